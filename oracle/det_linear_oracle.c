@@ -1,0 +1,195 @@
+/*
+ * CPU oracle for the deterministic fused-upcast linear layer  y = x * up(W_bf16)^T (+ b)
+ * (paper Eq. 2, design rules R1-R4).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, scalar, obviously-correct restatement of the
+ * reduction order; it shares no code with the CUDA path and is never on the product path.  Only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg may call it.
+ *
+ * The result of the method is not "the dot product": it is the outcome of one specific sequence of
+ * binary32 roundings (R1: every multiply-accumulate is one IEEE-754 FMA; R3: K is cut into contiguous
+ * segments whose partial sums are added in ascending order; R4: nothing depends on M).  The oracle
+ * therefore replays the sequence step by step, in the order family (V, L, P, seg_len):
+ *
+ *   - a segment [k_lo, k_hi) is walked in chunks of C = V*L elements, ascending;
+ *   - inside a chunk, "lane" l (0 <= l < L) owns the V consecutive elements  c + l*V + j, j = 0..V-1;
+ *   - element j of a lane is accumulated into that lane's sub-chain  p = j mod P, so there are L*P
+ *     leaves, leaf index  l*P + p; every accumulation is  a = fmaf(x, up(w), a)  starting from +0.0f;
+ *     elements at or beyond k_hi are skipped (not zero-filled);
+ *   - the L*P leaves are summed by a balanced binary tree, adjacent leaves first;
+ *   - the segment sums are added left to right in ascending segment order (R3, "fixed ascending
+ *     segment order"), and the bias, when present, is added last with one rounding (Eq. 2).
+ *
+ * The paper's own kernels are the member (V, L, P) = (1, 1, 1) of this family (strictly ascending k
+ * inside a segment, supplement C on R2).  The production constants are chosen by oracle.py.
+ *
+ * Parity status: the arithmetic is pinned by hand-traced examples, closed forms, an exact-rational
+ * re-implementation, an exact integer special case and an FP64 error bound (tests/test_oracle_*.py).
+ * The production constants themselves (V, L, P, bucket edge, split rule) are design choices that
+ * the paper does not print: for those, "parity unpinned" beyond the frozen definition.
+ *
+ * Build: gcc -O2 -std=c99 -ffp-contract=off -fno-fast-math -fopenmp -fPIC -shared (see build_oracle.py).
+ * fmaf() comes from libm and is correctly rounded; it is never emulated through double.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+#if defined(__x86_64__) || defined(__i386__)
+#include <xmmintrin.h>
+#define ORACLE_HAVE_MXCSR 1
+#endif
+
+#define ORACLE_MAX_LEAVES 4096
+
+/* up(): widen a BF16 bit pattern to binary32 by placing it in the high half (exact; Eq. 2). */
+float det_oracle_up(uint16_t h)
+{
+    uint32_t bits = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+/* Gradual underflow must be on: flush-to-zero / denormals-are-zero would change results for
+ * subnormal operands (R1 asks for IEEE-754 arithmetic).  Returns the previous control word. */
+static unsigned oracle_enter_ieee(void)
+{
+#ifdef ORACLE_HAVE_MXCSR
+    unsigned old = _mm_getcsr();
+    _mm_setcsr(old & ~(0x8000u | 0x0040u));   /* clear FTZ (bit 15) and DAZ (bit 6) */
+    return old;
+#else
+    return 0;
+#endif
+}
+static void oracle_leave_ieee(unsigned old)
+{
+#ifdef ORACLE_HAVE_MXCSR
+    _mm_setcsr(old);
+#else
+    (void)old;
+#endif
+}
+
+/* One output element y[m,n]: xrow = x[m,:], wrow = W[n,:], bias = &b[n] or NULL. */
+static float oracle_one(const float *xrow, const uint16_t *wrow, const float *bias,
+                        int64_t K, int V, int L, int P, int64_t seg_len)
+{
+    float a[ORACLE_MAX_LEAVES];
+    const int nleaf = L * P;
+    const int64_t C = (int64_t)V * L;
+    float t = 0.0f;
+    int64_t s = 0;
+    for (int64_t k_lo = 0; k_lo < K; k_lo += seg_len, ++s) {
+        int64_t k_hi = k_lo + seg_len;
+        if (k_hi > K) k_hi = K;
+        for (int i = 0; i < nleaf; ++i) a[i] = 0.0f;
+        for (int64_t c = k_lo; c < k_hi; c += C) {          /* chunks ascending */
+            for (int l = 0; l < L; ++l) {
+                for (int j = 0; j < V; ++j) {                /* elements ascending */
+                    int64_t k = c + (int64_t)l * V + j;
+                    if (k < k_hi) {
+                        int leaf = l * P + (j % P);
+                        a[leaf] = fmaf(xrow[k], det_oracle_up(wrow[k]), a[leaf]);
+                    }
+                }
+            }
+        }
+        for (int w = nleaf; w > 1; w /= 2)                   /* adjacent leaves first */
+            for (int i = 0; i < w / 2; ++i)
+                a[i] = a[2 * i] + a[2 * i + 1];
+        t = (s == 0) ? a[0] : (t + a[0]);                    /* ascending segment order */
+    }
+    return bias ? (t + *bias) : t;                           /* bias last, one rounding */
+}
+
+static int oracle_args_ok(int64_t M, int64_t N, int64_t K, int V, int L, int P, int64_t seg_len)
+{
+    if (M < 0 || N < 0 || K < 1 || V < 1 || L < 1 || P < 1 || seg_len < 1) return 0;
+    int nleaf = L * P;
+    if (nleaf > ORACLE_MAX_LEAVES || (nleaf & (nleaf - 1)) != 0) return 0;  /* balanced tree */
+    if (seg_len % ((int64_t)V * L) != 0 && seg_len < K) return 0;          /* segments start on chunk edges */
+    return 1;
+}
+
+/* Full problem.  x: [M,K] row-major FP32; W: [N,K] row-major BF16 bit patterns; b: [N] or NULL;
+ * y: [M,N] row-major.  Returns 0 on success, 1 on bad arguments. */
+int det_oracle_linear(const float *x, const uint16_t *W, const float *b, float *y,
+                      int64_t M, int64_t N, int64_t K,
+                      int V, int L, int P, int64_t seg_len, int nthreads)
+{
+    if (!oracle_args_ok(M, N, K, V, L, P, seg_len)) return 1;
+#ifdef _OPENMP
+    if (nthreads < 1) nthreads = omp_get_max_threads();
+#else
+    (void)nthreads;
+#endif
+    #pragma omp parallel num_threads(nthreads)
+    {
+        unsigned csr = oracle_enter_ieee();
+        #pragma omp for schedule(static)
+        for (int64_t n = 0; n < N; ++n)
+            for (int64_t m = 0; m < M; ++m)
+                y[m * N + n] = oracle_one(x + m * K, W + n * K, b ? b + n : NULL, K, V, L, P, seg_len);
+        oracle_leave_ieee(csr);
+    }
+    return 0;
+}
+
+/* Selected outputs only: out[i] = y[ms[i], ns[i]] (for full-size problems where the whole matrix
+ * would take too long). */
+int det_oracle_linear_sampled(const float *x, const uint16_t *W, const float *b,
+                              const int64_t *ms, const int64_t *ns, int64_t count, float *out,
+                              int64_t M, int64_t N, int64_t K,
+                              int V, int L, int P, int64_t seg_len, int nthreads)
+{
+    if (!oracle_args_ok(M, N, K, V, L, P, seg_len) || count < 0) return 1;
+    for (int64_t i = 0; i < count; ++i)
+        if (ms[i] < 0 || ms[i] >= M || ns[i] < 0 || ns[i] >= N) return 1;
+#ifdef _OPENMP
+    if (nthreads < 1) nthreads = omp_get_max_threads();
+#else
+    (void)nthreads;
+#endif
+    #pragma omp parallel num_threads(nthreads)
+    {
+        unsigned csr = oracle_enter_ieee();
+        #pragma omp for schedule(static)
+        for (int64_t i = 0; i < count; ++i)
+            out[i] = oracle_one(x + ms[i] * K, W + ns[i] * K, b ? b + ns[i] : NULL, K, V, L, P, seg_len);
+        oracle_leave_ieee(csr);
+    }
+    return 0;
+}
+
+/* Greedy argmax per row with the lower index winning a tie (the tie rule stated in the end-to-end
+ * determinism section).  -0.0 and +0.0 compare equal; if a row holds a NaN, the first NaN's index
+ * is returned (a NaN never occurs for finite inputs). */
+int det_oracle_argmax_rows(const float *y, int64_t M, int64_t N, int32_t *idx)
+{
+    if (M < 0 || N < 1) return 1;
+    for (int64_t m = 0; m < M; ++m) {
+        const float *row = y + m * N;
+        int64_t best = 0;
+        if (!isnan(row[0])) {
+            for (int64_t n = 1; n < N; ++n) {
+                if (isnan(row[n])) { best = n; break; }
+                if (row[n] > row[best]) best = n;
+            }
+        }
+        idx[m] = (int32_t)best;
+    }
+    return 0;
+}
+
+int det_oracle_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

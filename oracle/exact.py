@@ -1,0 +1,118 @@
+"""Exact-rational micro-oracle: the same reduction order, with every binary32 rounding carried out
+on Python `fractions.Fraction` values instead of by the CPU's FMA unit.
+
+TEST INFRASTRUCTURE ONLY.  It exists to check the C oracle's arithmetic (is fmaf really a single
+rounding? is the tree adjacent-first? are tails skipped?) with an implementation that shares
+neither language nor floating-point hardware with it.  Pure Python loops: tiny shapes only.
+
+Values are Python floats that are exactly representable in binary32 (a Python float can hold any
+binary32 value, including signed zeros and infinities).
+"""
+import math
+import struct
+from fractions import Fraction
+
+_MIN_EXP = -126          # exponent of the smallest normal binary32
+_MANT = 23               # explicit significand bits
+_MAX_FINITE = Fraction(2 ** 24 - 1, 1) * Fraction(2) ** (127 - 23)
+
+
+def bf16_bits_to_float(h: int) -> float:
+    """up(): the binary32 value whose bit pattern is h << 16 (Eq. 2's register upcast)."""
+    return struct.unpack("<f", struct.pack("<I", (h & 0xFFFF) << 16))[0]
+
+
+def round_to_binary32(q: Fraction) -> float:
+    """Round an exact rational to the nearest binary32, ties to even, gradual underflow,
+    overflow to infinity (IEEE-754 roundTiesToEven)."""
+    if q == 0:
+        return 0.0
+    sign = -1.0 if q < 0 else 1.0
+    a = -q if q < 0 else q
+    # e = floor(log2(a)), found exactly
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    elif Fraction(2) ** (e + 1) <= a:
+        e += 1
+    quantum = Fraction(2) ** (max(e, _MIN_EXP) - _MANT)
+    n = a / quantum
+    lo = n.numerator // n.denominator
+    rem = n - lo
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and (lo & 1)):
+        lo += 1
+    r = lo * quantum
+    # IEEE overflow rule: a value that rounds (with unbounded exponent) beyond the largest finite
+    # number becomes infinity
+    if r > _MAX_FINITE:
+        return sign * math.inf
+    return sign * float(r)       # exact: r has at most 24 significant bits; -0.0 when r == 0
+
+
+def _is_neg(v: float) -> bool:
+    return math.copysign(1.0, v) < 0
+
+
+def fma32(x: float, w: float, a: float) -> float:
+    """fusedMultiplyAdd in binary32: x*w + a with one rounding (rule R1)."""
+    if not (math.isfinite(x) and math.isfinite(w) and math.isfinite(a)):
+        raise ValueError("exact micro-oracle handles finite operands only")
+    q = Fraction(x) * Fraction(w) + Fraction(a)
+    if q != 0:
+        return round_to_binary32(q)        # a nonzero value that underflows keeps its own sign
+    # exact zero: -0 only when a zero product of negative sign meets a = -0; a cancellation of
+    # nonzero terms gives +0 under roundTiesToEven
+    prod_is_zero = (x == 0 or w == 0)
+    prod_neg = _is_neg(x) != _is_neg(w)
+    return -0.0 if (prod_is_zero and prod_neg and _is_neg(a)) else 0.0
+
+
+def add32(a: float, b: float) -> float:
+    """binary32 addition, one rounding."""
+    if not (math.isfinite(a) and math.isfinite(b)):
+        raise ValueError("exact micro-oracle handles finite operands only")
+    q = Fraction(a) + Fraction(b)
+    if q == 0:
+        zneg = (a == 0 and b == 0 and _is_neg(a) and _is_neg(b))
+        return -0.0 if zneg else 0.0
+    return round_to_binary32(q)
+
+
+def output(xrow, wrow, bias, V, L, P, seg_len):
+    """One output element.  xrow: binary32-representable floats; wrow: BF16 bit patterns (ints);
+    bias: float or None.  Follows the order family (V, L, P, seg_len): chunks of V*L elements
+    ascending, lane l owns V consecutive elements, element j feeds sub-chain j mod P, leaves are
+    tree-summed adjacent-first, segments are summed ascending, bias is added last."""
+    K = len(xrow)
+    assert len(wrow) == K
+    nleaf = L * P
+    assert nleaf & (nleaf - 1) == 0
+    C = V * L
+    t = None
+    k_lo = 0
+    while k_lo < K:
+        k_hi = min(K, k_lo + seg_len)
+        a = [0.0] * nleaf
+        c = k_lo
+        while c < k_hi:
+            for l in range(L):
+                for j in range(V):
+                    k = c + l * V + j
+                    if k < k_hi:
+                        leaf = l * P + (j % P)
+                        a[leaf] = fma32(xrow[k], bf16_bits_to_float(wrow[k]), a[leaf])
+            c += C
+        w = nleaf
+        while w > 1:
+            a = [add32(a[2 * i], a[2 * i + 1]) for i in range(w // 2)]
+            w //= 2
+        t = a[0] if t is None else add32(t, a[0])
+        k_lo += seg_len
+    return add32(t, bias) if bias is not None else t
+
+
+def linear(x, W_bits, b, V, L, P, seg_len):
+    """Whole (tiny) problem as nested lists: y[m][n]."""
+    return [[output(list(map(float, xr)), list(map(int, wr)), None if b is None else float(b[n]),
+                    V, L, P, seg_len)
+             for n, wr in enumerate(W_bits)] for xr in x]

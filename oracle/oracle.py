@@ -1,0 +1,169 @@
+"""Python face of the CPU oracle (ctypes over liboracle.so) and the oracle's own copy of the
+shape -> order-parameter rule.
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the benchmark's CPU-baseline
+leg; never by the product path, and it imports nothing from the CUDA package.
+
+The rule below restates, independently of the CUDA library's planner, how the reduction order is
+chosen from the problem shape alone (design rule R2: configuration is a pure function of (M, N, K);
+R3: the split is shape-pure; R4: inside the decode bucket nothing depends on M).  The tests assert
+that both sides arrive at the same parameters.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+from . import build_oracle
+
+ORDER_VERSION = 1
+
+#: segment boundaries fall on multiples of this many k elements in both buckets
+SEGMENT_GRANULE = 256
+#: decode bucket edge (R2/R4: "decode-shaped GEMMs (M <= 64)")
+DECODE_MAX_M = 64
+
+
+def _ceil_div(a: int, b: int) -> int:
+    return -(-a // b)
+
+
+def split_request(M: int, N: int, K: int) -> int:
+    """Requested number of K segments before clamping to what K allows.
+
+    Decode (never reads M, rule R4): 1 when N >= 4096 (enough rows to fill the machine, like the
+    paper's lm_head "prefers no split"); otherwise the smallest power of two with N*S >= 4096.
+    Prefill: the smallest power of two S <= 16 with tiles*S >= 1024 where tiles counts 128x128
+    output tiles, never cutting a segment below 512 elements.
+    """
+    if M <= DECODE_MAX_M:
+        s = 1
+        while N * s < 4096:
+            s *= 2
+        return s
+    tiles = _ceil_div(M, 128) * _ceil_div(N, 128)
+    s = 1
+    while s < 16 and tiles * s < 1024 and K // (2 * s) >= 512:
+        s *= 2
+    return s
+
+
+def order_params(M: int, N: int, K: int) -> dict:
+    """Order parameters for a problem shape: bucket, (V, L, P), seg_len and the segment count S."""
+    if min(M, N, K) < 1:
+        raise ValueError("M, N, K must be >= 1")
+    if M <= DECODE_MAX_M:
+        bucket, V, L, P = "decode", 4, 32, 2
+    else:
+        bucket, V, L, P = "prefill", 2, 1, 2
+    s_req = split_request(M, N, K)
+    n_gran = _ceil_div(K, SEGMENT_GRANULE)
+    gran_per_seg = _ceil_div(n_gran, min(s_req, n_gran))
+    seg_len = SEGMENT_GRANULE * gran_per_seg
+    S = _ceil_div(n_gran, gran_per_seg)
+    return {"bucket": bucket, "V": V, "L": L, "P": P, "seg_len": seg_len, "S": S,
+            "order_version": ORDER_VERSION}
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        path = build_oracle.build()
+        L = ctypes.CDLL(path)
+        i64, i32, p = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p
+        L.det_oracle_linear.argtypes = [p, p, p, p, i64, i64, i64, i32, i32, i32, i64, i32]
+        L.det_oracle_linear.restype = i32
+        L.det_oracle_linear_sampled.argtypes = [p, p, p, p, p, i64, p, i64, i64, i64,
+                                                i32, i32, i32, i64, i32]
+        L.det_oracle_linear_sampled.restype = i32
+        L.det_oracle_argmax_rows.argtypes = [p, i64, i64, p]
+        L.det_oracle_argmax_rows.restype = i32
+        L.det_oracle_up.argtypes = [ctypes.c_uint16]
+        L.det_oracle_up.restype = ctypes.c_float
+        L.det_oracle_threads.restype = i32
+        _lib = L
+    return _lib
+
+
+def _f32(a, shape):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    assert a.shape == shape, (a.shape, shape)
+    return a
+
+
+def _bf16_bits(W, shape):
+    W = np.ascontiguousarray(W)
+    assert W.dtype == np.uint16, "W must be given as BF16 bit patterns (uint16)"
+    assert W.shape == shape, (W.shape, shape)
+    return W
+
+
+def _resolve(M, N, K, params):
+    prm = order_params(M, N, K) if params is None else params
+    return int(prm["V"]), int(prm["L"]), int(prm["P"]), int(prm["seg_len"])
+
+
+def linear(x, W_bits, b=None, params=None, threads=0):
+    """y = x . up(W)^T (+ b) in the frozen order.  x [M,K] float32, W_bits [N,K] uint16 (BF16 bit
+    patterns), b [N] float32 or None.  `params` overrides the shape-derived order (for the scaled-
+    down hand examples)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    M, K = x.shape
+    N = W_bits.shape[0]
+    W_bits = _bf16_bits(W_bits, (N, K))
+    V, L, P, seg_len = _resolve(M, N, K, params)
+    y = np.empty((M, N), dtype=np.float32)
+    bp = None
+    if b is not None:
+        b = _f32(b, (N,))
+        bp = b.ctypes.data
+    rc = lib().det_oracle_linear(x.ctypes.data, W_bits.ctypes.data, bp, y.ctypes.data,
+                                 M, N, K, V, L, P, seg_len, threads)
+    if rc != 0:
+        raise ValueError("det_oracle_linear rejected its arguments")
+    return y
+
+
+def linear_sampled(x, W_bits, b, ms, ns, params=None, threads=0):
+    """Selected outputs y[ms[i], ns[i]] of the same computation."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    M, K = x.shape
+    N = W_bits.shape[0]
+    W_bits = _bf16_bits(W_bits, (N, K))
+    V, L, P, seg_len = _resolve(M, N, K, params)
+    ms = np.ascontiguousarray(ms, dtype=np.int64)
+    ns = np.ascontiguousarray(ns, dtype=np.int64)
+    out = np.empty(ms.shape[0], dtype=np.float32)
+    bp = None
+    if b is not None:
+        b = _f32(b, (N,))
+        bp = b.ctypes.data
+    rc = lib().det_oracle_linear_sampled(x.ctypes.data, W_bits.ctypes.data, bp, ms.ctypes.data,
+                                         ns.ctypes.data, ms.shape[0], out.ctypes.data,
+                                         M, N, K, V, L, P, seg_len, threads)
+    if rc != 0:
+        raise ValueError("det_oracle_linear_sampled rejected its arguments")
+    return out
+
+
+def argmax_rows(y):
+    """Index of the row maximum, lowest index on ties."""
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    M, N = y.shape
+    idx = np.empty(M, dtype=np.int32)
+    rc = lib().det_oracle_argmax_rows(y.ctypes.data, M, N, idx.ctypes.data)
+    if rc != 0:
+        raise ValueError("det_oracle_argmax_rows rejected its arguments")
+    return idx
+
+
+def up(h: int) -> float:
+    return float(lib().det_oracle_up(int(h) & 0xFFFF))
+
+
+def threads() -> int:
+    """Threads the oracle uses by default (bounded by the process's CPU affinity)."""
+    return min(int(lib().det_oracle_threads()), len(os.sched_getaffinity(0)))
