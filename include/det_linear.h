@@ -1,0 +1,149 @@
+/*
+ * det_linear.h -- C ABI of the deterministic fused-upcast linear layer for NVIDIA B200 (sm_100a).
+ *
+ *     y = x * up(W_bf16)^T (+ b)                                            (paper Eq. 2)
+ *
+ * FP32 activations, BF16 weights read once from HBM and widened to FP32 in registers, IEEE-754
+ * FP32 fused multiply-add accumulation on the CUDA cores (design rule R1: never tensor cores), in
+ * a reduction order that is a pure function of the problem shape (M, N, K) (rules R2-R4): the bits
+ * of y do not depend on the SM count, the grid, the stream, co-scheduled work or, inside the
+ * decode bucket (M <= 64), on M.
+ *
+ * Reduction order, version 1 (what "the same bits" means):
+ *   bucket   = decode if M <= 64, else prefill                                  (R2, R4)
+ *   decode : V = 4, L = 32, P = 2        prefill: V = 2, L = 1, P = 2
+ *   K is cut into S contiguous segments of seg_len elements (a multiple of 256; only the last
+ *   may be short); S is shape-pure and, for decode, independent of M               (R3, R4)
+ *   inside a segment, chunks of V*L elements are walked in ascending k; "lane" l owns the V
+ *   consecutive elements c + l*V + j; element j is accumulated with one fmaf into the lane's
+ *   sub-chain j mod P, starting from +0.0f; elements beyond the segment end are skipped;
+ *   the L*P leaves are summed by a balanced tree, adjacent leaves first;
+ *   segment sums are added in ascending segment order (R3, no atomics);
+ *   the bias, when given, is added last with a single rounding                    (Eq. 2).
+ *
+ * All functions return a status or NULL and never throw, abort or synchronise the device unless
+ * stated.  Pointers named "device" must be device memory of the current CUDA device; "host" means
+ * ordinary (preferably pinned) host memory.  The library requires compute capability 10.x; on any
+ * other device plan creation fails with DET_ERR_ARCH (there is no fallback path).
+ */
+#ifndef DET_LINEAR_H
+#define DET_LINEAR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DET_API __attribute__((visibility("default")))
+#else
+#define DET_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct det_linear_plan det_linear_plan_t;   /* opaque, owned by the library */
+
+typedef enum {
+    DET_OK = 0,
+    DET_ERR_INVALID_ARG = 1,        /* NULL pointer, non-positive size, buffer too small          */
+    DET_ERR_UNSUPPORTED_SHAPE = 2,  /* a dimension exceeds what the kernels index (see below)     */
+    DET_ERR_ALIGNMENT = 3,          /* reserved: misaligned buffers take the generic kernel       */
+    DET_ERR_ALLOC = 4,              /* device or host allocation failed                           */
+    DET_ERR_CUDA = 5,               /* a CUDA call failed; det_last_error() has the message       */
+    DET_ERR_DEVICE_TIMEOUT = 6,     /* a kernel gave up a bounded wait (see det_linear_plan_check)*/
+    DET_ERR_ARCH = 7                /* current device is not sm_100                               */
+} det_status_t;
+
+/* Order parameters of a shape; filled by det_linear_plan_params / det_linear_plan_get_params. */
+typedef struct {
+    int64_t M, N, K;
+    int32_t bucket;          /* 0 = decode (M <= 64), 1 = prefill                                   */
+    int32_t V, L, P;         /* order family parameters (see the header comment)                    */
+    int64_t seg_len;         /* K elements per segment                                              */
+    int32_t S;               /* number of segments, = ceil(K / seg_len)                             */
+    int32_t order_version;   /* version of the order definition, 1                                  */
+    int32_t kernel;          /* 0 generic, 1 decode (TMA pipeline), 2 prefill tile kernel           */
+    int32_t reserved;
+    uint64_t workspace_bytes;/* split-K partials: 4*S*M*N bytes when S > 1, else 0                  */
+} det_linear_params_t;
+
+/*
+ * Shape -> order parameters (rule R2: "compile-time constants selected by a pure function of the
+ * problem shape"; R3: the split is shape-pure; R4: decode parameters never read M).  Pure host
+ * function: touches no device, allocates nothing.  M, N, K >= 1 and each < 2^31, M*N < 2^40.
+ * The `kernel` field reports the kernel for 16-byte aligned buffers.
+ */
+DET_API det_status_t det_linear_plan_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* out);
+
+/*
+ * Create a plan for y[M,N] = x[M,K] * up(W[N,K])^T (+ b[N]) on the current device.  Allocates the
+ * split-K partials workspace (device) when S > 1.  Returns NULL on failure (det_last_error()).
+ * A plan may be used from one stream at a time: its workspace is not re-entrant; make one plan
+ * per stream for concurrent use.  Destroy with det_linear_plan_destroy.
+ */
+DET_API det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K);
+
+/*
+ * Enqueue the computation on `stream` (a cudaStream_t; NULL = the legacy default stream) and
+ * return without synchronising.  Eq. 2 with the order above; split-K partials, if any, are
+ * combined by a second fixed-order pass (R3), never by atomics.
+ *   x : device, FP32, [M,K] row-major (row pitch K)
+ *   W : device, BF16 bit patterns, [N,K] row-major (row pitch K): one weight row per output column
+ *   b : device, FP32, [N], or NULL for no bias (then no final add happens at all)
+ *   y : device, FP32, [M,N] row-major; overwritten; must not overlap the inputs
+ * Buffers stay owned by the caller and must stay valid until the stream reaches the end of the
+ * work.  The fast kernels need K % 8 == 0 and 16-byte aligned x, W, y; anything else runs a
+ * slower generic kernel that produces the same bits.  Errors: DET_ERR_INVALID_ARG for NULL
+ * arguments, DET_ERR_CUDA if a launch fails.  Nothing is launched when an error is returned.
+ */
+DET_API det_status_t det_linear_run(const det_linear_plan_t* plan, const float* x, const uint16_t* W,
+                            const float* b, float* y, void* stream);
+
+/*
+ * End-to-end variant with HOST activations: copies x (host, [M,K]) to a plan-owned device buffer,
+ * runs the same kernels, copies y back to y_host (host, [M,N]) and waits for the stream.  W and b
+ * stay device-resident (they are the model's parameters).  The staging buffers are allocated on
+ * first use.  Synchronises `stream` before returning.
+ */
+DET_API det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, const uint16_t* W,
+                                 const float* b, float* y_host, void* stream);
+
+/*
+ * Synchronise `stream` and report whether any kernel launched through this plan gave up a bounded
+ * device-side wait (every wait on a TMA completion barrier is limited; on expiry the kernel
+ * records the fact and returns instead of spinning).  DET_OK, DET_ERR_DEVICE_TIMEOUT or
+ * DET_ERR_CUDA.  The record is cleared by the call.
+ */
+DET_API det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream);
+
+/* Copy the plan's order parameters to *out. */
+DET_API det_status_t det_linear_plan_get_params(const det_linear_plan_t* plan, det_linear_params_t* out);
+
+/* Write a JSON description (bucket, V, L, P, S, seg_len, order_version, kernel, workspace_bytes)
+ * to buf (at most n bytes including the terminator).  DET_ERR_INVALID_ARG if it does not fit. */
+DET_API det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, size_t n);
+
+/* Free the plan and everything it owns.  NULL is ignored.  The caller must make sure no work
+ * using the plan is still running. */
+DET_API void det_linear_plan_destroy(det_linear_plan_t* plan);
+
+/*
+ * Greedy argmax per row with the LOWER index winning a tie (the tie rule the paper states for
+ * greedy decoding): idx[m] = min{ n : y[m,n] = max_n y[m,n] }.  -0.0 and +0.0 compare equal; a
+ * row containing NaN returns the index of its first NaN.
+ *   y : device FP32 [M,N] row-major;  idx : device int32 [M].  1 <= N < 2^31, M >= 1.
+ * Enqueued on `stream`, no synchronisation.  Exact (comparisons only), so it is order-free.
+ */
+DET_API det_status_t det_argmax_rows(const float* y, int64_t M, int64_t N, int32_t* idx, void* stream);
+
+/* Message of the last error on the calling thread ("" if none).  Never NULL. */
+DET_API const char* det_last_error(void);
+
+/* Version of the reduction-order definition implemented by this library (currently 1). */
+DET_API int det_order_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DET_LINEAR_H */

@@ -1,0 +1,44 @@
+/*
+ * det_linear_test.h -- test-only exports of the det_linear library.  Nothing here changes the
+ * arithmetic: the hooks select among kernels and launch geometries that must all produce the same
+ * bits (tile sizes, warp counts, pipeline depth and grid size are numerically inert: supplement C
+ * on rule R2), and create streams restricted to a subset of the SMs so that tests can check that
+ * the output does not depend on the SM count (rule R3: "independent of the device, its SM count,
+ * and grid scheduling").  The paper has no counterpart for these functions.
+ */
+#ifndef DET_LINEAR_TEST_H
+#define DET_LINEAR_TEST_H
+
+#include "det_linear.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Force the kernel a plan uses: 0 generic, 1 decode pipeline, 2 prefill tile kernel, -1 automatic.
+ * DET_ERR_INVALID_ARG when the kernel cannot serve the plan's bucket. */
+DET_API det_status_t det_test_plan_force_kernel(det_linear_plan_t* plan, int kernel);
+
+/* Limit the number of thread blocks the plan's persistent kernels launch (0 = automatic, i.e.
+ * derived from the SM count).  Only the schedule changes. */
+DET_API det_status_t det_test_plan_set_max_blocks(det_linear_plan_t* plan, int max_blocks);
+
+/* Select a tile configuration variant of the plan's kernel (0 = automatic). Only the schedule
+ * changes. DET_ERR_INVALID_ARG if the variant does not exist for this plan. */
+DET_API det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant);
+
+/*
+ * Create a CUDA green context holding (at least) `sm_count` SMs of the current device and a
+ * stream on it.  *stream_out receives a cudaStream_t usable with det_linear_run; *handle_out an
+ * opaque handle for det_test_green_stream_destroy; *sm_granted the number of SMs in the
+ * partition.  DET_ERR_CUDA if the driver refuses (the caller should then fall back to other
+ * invariance checks).
+ */
+DET_API det_status_t det_test_green_stream_create(int sm_count, void** stream_out, void** handle_out,
+                                          int* sm_granted);
+DET_API void det_test_green_stream_destroy(void* handle);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DET_LINEAR_TEST_H */

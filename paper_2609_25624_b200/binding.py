@@ -1,0 +1,219 @@
+"""Thin Python binding of libdet_linear.so (ctypes): argument marshalling only.
+
+Every function has the name of the C entry point it calls (include/det_linear.h) minus nothing:
+`det_linear_plan`, `det_linear_run`, ...  Tensors are torch CUDA tensors; only their data pointers,
+shapes and the current stream cross the boundary.  There is no CPU fallback: if the shared library
+is missing or cannot be loaded, importing symbols from here raises.
+"""
+import ctypes
+import json
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdet_linear.so")
+
+DET_OK = 0
+STATUS_NAMES = {0: "DET_OK", 1: "DET_ERR_INVALID_ARG", 2: "DET_ERR_UNSUPPORTED_SHAPE", 3: "DET_ERR_ALIGNMENT",
+                4: "DET_ERR_ALLOC", 5: "DET_ERR_CUDA", 6: "DET_ERR_DEVICE_TIMEOUT", 7: "DET_ERR_ARCH"}
+
+
+class DetLinearError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+class Params(ctypes.Structure):
+    """Mirror of det_linear_params_t."""
+    _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("bucket", ctypes.c_int32), ("V", ctypes.c_int32), ("L", ctypes.c_int32), ("P", ctypes.c_int32),
+                ("seg_len", ctypes.c_int64), ("S", ctypes.c_int32), ("order_version", ctypes.c_int32),
+                ("kernel", ctypes.c_int32), ("reserved", ctypes.c_int32), ("workspace_bytes", ctypes.c_uint64)]
+
+    def as_dict(self):
+        return {"bucket": "decode" if self.bucket == 0 else "prefill", "V": self.V, "L": self.L, "P": self.P,
+                "seg_len": self.seg_len, "S": self.S, "order_version": self.order_version}
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libdet_linear.so (once).  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_25624_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        p, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        L.det_linear_plan_params.argtypes = [i64, i64, i64, ctypes.POINTER(Params)]
+        L.det_linear_plan_params.restype = i32
+        L.det_linear_plan.argtypes = [i64, i64, i64]
+        L.det_linear_plan.restype = p
+        L.det_linear_run.argtypes = [p, p, p, p, p, p]
+        L.det_linear_run.restype = i32
+        L.det_linear_run_host.argtypes = [p, p, p, p, p, p]
+        L.det_linear_run_host.restype = i32
+        L.det_linear_plan_check.argtypes = [p, p]
+        L.det_linear_plan_check.restype = i32
+        L.det_linear_plan_get_params.argtypes = [p, ctypes.POINTER(Params)]
+        L.det_linear_plan_get_params.restype = i32
+        L.det_linear_plan_describe.argtypes = [p, ctypes.c_char_p, ctypes.c_size_t]
+        L.det_linear_plan_describe.restype = i32
+        L.det_linear_plan_destroy.argtypes = [p]
+        L.det_linear_plan_destroy.restype = None
+        L.det_argmax_rows.argtypes = [p, i64, i64, p, p]
+        L.det_argmax_rows.restype = i32
+        L.det_last_error.restype = ctypes.c_char_p
+        L.det_order_version.restype = i32
+        L.det_test_plan_force_kernel.argtypes = [p, i32]
+        L.det_test_plan_force_kernel.restype = i32
+        L.det_test_plan_set_max_blocks.argtypes = [p, i32]
+        L.det_test_plan_set_max_blocks.restype = i32
+        L.det_test_plan_set_variant.argtypes = [p, i32]
+        L.det_test_plan_set_variant.restype = i32
+        L.det_test_green_stream_create.argtypes = [i32, ctypes.POINTER(p), ctypes.POINTER(p), ctypes.POINTER(i32)]
+        L.det_test_green_stream_create.restype = i32
+        L.det_test_green_stream_destroy.argtypes = [p]
+        L.det_test_green_stream_destroy.restype = None
+        _lib = L
+    return _lib
+
+
+def _check(status):
+    if status != DET_OK:
+        raise DetLinearError(status, det_last_error())
+
+
+def det_last_error() -> str:
+    return lib().det_last_error().decode()
+
+
+def det_order_version() -> int:
+    return int(lib().det_order_version())
+
+
+def det_linear_plan_params(M: int, N: int, K: int) -> Params:
+    out = Params()
+    _check(lib().det_linear_plan_params(M, N, K, ctypes.byref(out)))
+    return out
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+class Plan:
+    """Owner of a det_linear_plan_t*."""
+
+    def __init__(self, M: int, N: int, K: int):
+        self.M, self.N, self.K = int(M), int(N), int(K)
+        self._h = lib().det_linear_plan(self.M, self.N, self.K)
+        if not self._h:
+            raise DetLinearError(-1, det_last_error())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().det_linear_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self):
+        return self._h
+
+
+def det_linear_plan(M: int, N: int, K: int) -> Plan:
+    return Plan(M, N, K)
+
+
+def det_linear_plan_destroy(plan: Plan) -> None:
+    plan.close()
+
+
+def det_linear_plan_get_params(plan: Plan) -> Params:
+    out = Params()
+    _check(lib().det_linear_plan_get_params(plan.handle, ctypes.byref(out)))
+    return out
+
+
+def det_linear_plan_describe(plan: Plan) -> dict:
+    buf = ctypes.create_string_buffer(512)
+    _check(lib().det_linear_plan_describe(plan.handle, buf, 512))
+    return json.loads(buf.value.decode())
+
+
+def _expect(t, dtype, shape, name):
+    if not t.is_cuda or t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise ValueError(f"{name}: need a contiguous CUDA tensor of dtype {dtype} and shape {tuple(shape)}, "
+                         f"got {t.dtype} {tuple(t.shape)} cuda={t.is_cuda}")
+
+
+def det_linear_run(plan: Plan, x, W, b, y, stream=None) -> None:
+    """Enqueue y = x . up(W)^T (+ b) on `stream` (default: torch's current stream)."""
+    _expect(x, torch.float32, (plan.M, plan.K), "x")
+    _expect(W, torch.bfloat16, (plan.N, plan.K), "W")
+    _expect(y, torch.float32, (plan.M, plan.N), "y")
+    if b is not None:
+        _expect(b, torch.float32, (plan.N,), "b")
+    _check(lib().det_linear_run(plan.handle, x.data_ptr(), W.data_ptr(), b.data_ptr() if b is not None else None,
+                                y.data_ptr(), _stream_ptr(stream)))
+
+
+def det_linear_run_host(plan: Plan, x_host, W, b, y_host, stream=None) -> None:
+    """x_host / y_host are (pinned) CPU tensors; W, b are CUDA tensors.  Synchronises the stream."""
+    for t, shape, name in ((x_host, (plan.M, plan.K), "x_host"), (y_host, (plan.M, plan.N), "y_host")):
+        if t.is_cuda or t.dtype != torch.float32 or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError(f"{name}: need a contiguous CPU float32 tensor of shape {shape}")
+    _expect(W, torch.bfloat16, (plan.N, plan.K), "W")
+    if b is not None:
+        _expect(b, torch.float32, (plan.N,), "b")
+    _check(lib().det_linear_run_host(plan.handle, x_host.data_ptr(), W.data_ptr(),
+                                     b.data_ptr() if b is not None else None, y_host.data_ptr(),
+                                     _stream_ptr(stream)))
+
+
+def det_linear_plan_check(plan: Plan, stream=None) -> None:
+    _check(lib().det_linear_plan_check(plan.handle, _stream_ptr(stream)))
+
+
+def det_argmax_rows(y, idx, stream=None) -> None:
+    M, N = y.shape
+    _expect(y, torch.float32, (M, N), "y")
+    _expect(idx, torch.int32, (M,), "idx")
+    _check(lib().det_argmax_rows(y.data_ptr(), M, N, idx.data_ptr(), _stream_ptr(stream)))
+
+
+# ---- test-only exports (include/det_linear_test.h) ------------------------------------------
+def det_test_plan_force_kernel(plan: Plan, kernel: int) -> None:
+    _check(lib().det_test_plan_force_kernel(plan.handle, kernel))
+
+
+def det_test_plan_set_max_blocks(plan: Plan, max_blocks: int) -> None:
+    _check(lib().det_test_plan_set_max_blocks(plan.handle, max_blocks))
+
+
+def det_test_plan_set_variant(plan: Plan, variant: int) -> None:
+    _check(lib().det_test_plan_set_variant(plan.handle, variant))
+
+
+def det_test_green_stream_create(sm_count: int):
+    """Returns (stream_ptr:int, handle, sm_granted)."""
+    st, h, g = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_int(0)
+    _check(lib().det_test_green_stream_create(sm_count, ctypes.byref(st), ctypes.byref(h), ctypes.byref(g)))
+    return st.value, h, g.value
+
+
+def det_test_green_stream_destroy(handle) -> None:
+    lib().det_test_green_stream_destroy(handle)

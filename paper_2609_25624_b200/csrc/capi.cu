@@ -1,0 +1,345 @@
+// C ABI of libdet_linear: argument checks, plan life cycle, kernel dispatch.  Host code only.
+#include "internal.h"
+#include "det_linear_test.h"
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+namespace detlin {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+}
+
+static det_status_t cuda_fail(const char* what, cudaError_t e)
+{
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    return DET_ERR_CUDA;
+}
+
+// Driver entry points are looked up at run time so that the library loads on machines without
+// a driver (the build check and the symbol test run on CPU-only hosts).
+template <typename Fn>
+static Fn driver_fn(const char* name)
+{
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint(name, &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+        return nullptr;
+    return reinterpret_cast<Fn>(fn);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D row-major tensor [rows, cols] of `elem_bytes`-wide elements, box [box_rows, box_cols].
+static bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t rows,
+                      uint64_t cols, uint32_t box_rows, uint32_t box_cols, CUtensorMapL2promotion promo)
+{
+    static EncodeTiledFn encode = driver_fn<EncodeTiledFn>("cuTensorMapEncodeTiled");
+    if (!encode) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return false; }
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_NONE, promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r); return false; }
+    return true;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static det_status_t run_device(det_linear_plan_t* plan, const float* x, const uint16_t* W, const float* b, float* y,
+                               cudaStream_t stream)
+{
+    const det_linear_params_t& p = plan->prm;
+    LaunchArgs a{};
+    a.x = x; a.W = W; a.b = b; a.y = y;
+    a.partials = plan->partials;
+    a.M = p.M; a.N = p.N; a.K = p.K;
+    a.seg_len = p.seg_len; a.S = p.S;
+    a.stream = stream;
+    a.status = plan->status;
+    a.sm_count = plan->sm_count;
+    a.max_blocks = plan->max_blocks;
+    a.variant = plan->variant;
+
+    int kernel = plan->forced_kernel >= 0 ? plan->forced_kernel : p.kernel;
+    const bool fast_ok = (p.K % 8 == 0) && aligned16(x) && aligned16(W) && aligned16(y);
+    if (!fast_ok) kernel = kKernelGeneric;
+
+    cudaError_t e = cudaSuccess;
+    if (kernel == kKernelDecode) {
+        DecodeConfig cfg;
+        if (!decode_config_for(p.M, p.N, p.K, plan->variant, &cfg)) {
+            set_error("run: no decode configuration for this shape/variant");
+            return DET_ERR_INVALID_ARG;
+        }
+        if (plan->map_w_ptr != W || plan->map_x_ptr != x || plan->map_cfg_id != cfg.id) {
+            if (!encode_2d(&plan->map_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)p.N, (uint64_t)p.K,
+                           (uint32_t)cfg.rt, (uint32_t)cfg.kc, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+                return DET_ERR_CUDA;
+            if (!encode_2d(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, x, (uint64_t)p.M, (uint64_t)p.K,
+                           (uint32_t)(cfg.mt * cfg.wm), (uint32_t)cfg.kc, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+                return DET_ERR_CUDA;
+            plan->map_w_ptr = W; plan->map_x_ptr = x; plan->map_cfg_id = cfg.id;
+        }
+        e = launch_decode(a, &plan->map_w, &plan->map_x);
+    } else if (kernel == kKernelPrefill) {
+        e = launch_prefill(a);
+    } else {
+        e = launch_generic(a, p.bucket);
+    }
+    if (e != cudaSuccess) return cuda_fail("kernel launch", e);
+    return DET_OK;
+}
+
+}  // namespace detlin
+
+using namespace detlin;
+
+extern "C" {
+
+det_status_t det_linear_plan_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* out)
+{
+    return fill_params(M, N, K, out);
+}
+
+det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K)
+{
+    det_linear_params_t prm;
+    if (fill_params(M, N, K, &prm) != DET_OK) return nullptr;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { cuda_fail("cudaGetDevice", e); return nullptr; }
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) { cuda_fail("cudaGetDeviceProperties", e); return nullptr; }
+    if (prop.major != 10) {
+        set_error("plan: device %d is sm_%d%d; this library is built for sm_100a only (no fallback)", dev, prop.major,
+                  prop.minor);
+        return nullptr;
+    }
+    det_linear_plan_t* plan = new (std::nothrow) det_linear_plan_t();
+    if (!plan) { set_error("plan: host allocation failed"); return nullptr; }
+    memset(plan, 0, sizeof *plan);
+    plan->prm = prm;
+    plan->device = dev;
+    plan->sm_count = prop.multiProcessorCount;
+    plan->forced_kernel = -1;
+    plan->map_cfg_id = -1;
+    e = cudaMalloc(&plan->status, sizeof(DeviceStatus));
+    if (e == cudaSuccess) e = cudaMemset(plan->status, 0, sizeof(DeviceStatus));
+    if (e == cudaSuccess && prm.workspace_bytes) e = cudaMalloc(&plan->partials, prm.workspace_bytes);
+    if (e != cudaSuccess) {
+        set_error("plan: device allocation of %llu bytes failed: %s", (unsigned long long)prm.workspace_bytes,
+                  cudaGetErrorString(e));
+        cudaGetLastError();
+        det_linear_plan_destroy(plan);
+        return nullptr;
+    }
+    return plan;
+}
+
+det_status_t det_linear_run(const det_linear_plan_t* plan, const float* x, const uint16_t* W, const float* b, float* y,
+                            void* stream)
+{
+    if (!plan || !x || !W || !y) { set_error("run: plan, x, W and y must not be NULL"); return DET_ERR_INVALID_ARG; }
+    // the plan's tensor-map cache is the only state a run touches
+    return run_device(const_cast<det_linear_plan_t*>(plan), x, W, b, y, static_cast<cudaStream_t>(stream));
+}
+
+det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, const uint16_t* W, const float* b,
+                                 float* y_host, void* stream)
+{
+    if (!plan || !x_host || !W || !y_host) {
+        set_error("run_host: plan, x_host, W and y_host must not be NULL");
+        return DET_ERR_INVALID_ARG;
+    }
+    const det_linear_params_t& p = plan->prm;
+    const size_t xb = (size_t)p.M * p.K * 4, yb = (size_t)p.M * p.N * 4;
+    cudaError_t e;
+    if (!plan->x_stage) {
+        e = cudaMalloc(&plan->x_stage, xb);
+        if (e == cudaSuccess) e = cudaMalloc(&plan->y_stage, yb);
+        if (e != cudaSuccess) { set_error("run_host: staging allocation failed: %s", cudaGetErrorString(e)); cudaGetLastError(); return DET_ERR_ALLOC; }
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    e = cudaMemcpyAsync(plan->x_stage, x_host, xb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail("run_host: copy of x", e);
+    det_status_t s = run_device(plan, plan->x_stage, W, b, plan->y_stage, st);
+    if (s != DET_OK) return s;
+    e = cudaMemcpyAsync(y_host, plan->y_stage, yb, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail("run_host: copy of y", e);
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail("run_host: synchronise", e);
+    return DET_OK;
+}
+
+det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream)
+{
+    if (!plan) { set_error("check: plan is NULL"); return DET_ERR_INVALID_ARG; }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceStatus h{};
+    cudaError_t e = cudaMemcpyAsync(&h, plan->status, sizeof h, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(plan->status, 0, sizeof h, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail("check", e);
+    if (h.timeout_flag) {
+        set_error("check: a kernel gave up a bounded wait (site %u)", h.where);
+        return DET_ERR_DEVICE_TIMEOUT;
+    }
+    return DET_OK;
+}
+
+det_status_t det_linear_plan_get_params(const det_linear_plan_t* plan, det_linear_params_t* out)
+{
+    if (!plan || !out) { set_error("get_params: NULL argument"); return DET_ERR_INVALID_ARG; }
+    *out = plan->prm;
+    return DET_OK;
+}
+
+det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, size_t n)
+{
+    if (!plan || !buf || n == 0) { set_error("describe: NULL argument"); return DET_ERR_INVALID_ARG; }
+    const det_linear_params_t& p = plan->prm;
+    static const char* kn[] = {"generic", "decode", "prefill"};
+    int w = snprintf(buf, n,
+                     "{\"M\": %lld, \"N\": %lld, \"K\": %lld, \"bucket\": \"%s\", \"V\": %d, \"L\": %d, \"P\": %d, "
+                     "\"seg_len\": %lld, \"S\": %d, \"order_version\": %d, \"kernel\": \"%s\", \"workspace_bytes\": %llu}",
+                     (long long)p.M, (long long)p.N, (long long)p.K, p.bucket == 0 ? "decode" : "prefill", p.V, p.L, p.P,
+                     (long long)p.seg_len, p.S, p.order_version, kn[p.kernel], (unsigned long long)p.workspace_bytes);
+    if (w < 0 || (size_t)w >= n) { set_error("describe: buffer too small (%d bytes needed)", w + 1); return DET_ERR_INVALID_ARG; }
+    return DET_OK;
+}
+
+void det_linear_plan_destroy(det_linear_plan_t* plan)
+{
+    if (!plan) return;
+    if (plan->partials) cudaFree(plan->partials);
+    if (plan->status) cudaFree(plan->status);
+    if (plan->x_stage) cudaFree(plan->x_stage);
+    if (plan->y_stage) cudaFree(plan->y_stage);
+    delete plan;
+}
+
+det_status_t det_argmax_rows(const float* y, int64_t M, int64_t N, int32_t* idx, void* stream)
+{
+    if (!y || !idx) { set_error("argmax: NULL argument"); return DET_ERR_INVALID_ARG; }
+    if (M < 1 || N < 1 || N >= ((int64_t)1 << 31)) { set_error("argmax: need M >= 1 and 1 <= N < 2^31"); return DET_ERR_INVALID_ARG; }
+    cudaError_t e = launch_argmax(y, M, N, idx, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail("argmax launch", e);
+    return DET_OK;
+}
+
+const char* det_last_error(void) { return g_err; }
+
+int det_order_version(void) { return kOrderVersion; }
+
+// ---------------------------------------------------------------------------------------------
+// test-only exports
+// ---------------------------------------------------------------------------------------------
+det_status_t det_test_plan_force_kernel(det_linear_plan_t* plan, int kernel)
+{
+    if (!plan) { set_error("force_kernel: plan is NULL"); return DET_ERR_INVALID_ARG; }
+    if (kernel < -1 || kernel > 2 || (kernel == kKernelDecode && plan->prm.bucket != 0) ||
+        (kernel == kKernelPrefill && plan->prm.bucket != 1)) {
+        set_error("force_kernel: kernel %d cannot serve this plan's bucket", kernel);
+        return DET_ERR_INVALID_ARG;
+    }
+    plan->forced_kernel = kernel;
+    return DET_OK;
+}
+
+det_status_t det_test_plan_set_max_blocks(det_linear_plan_t* plan, int max_blocks)
+{
+    if (!plan || max_blocks < 0) { set_error("set_max_blocks: bad argument"); return DET_ERR_INVALID_ARG; }
+    plan->max_blocks = max_blocks;
+    return DET_OK;
+}
+
+det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
+{
+    if (!plan || variant < 0) { set_error("set_variant: bad argument"); return DET_ERR_INVALID_ARG; }
+    if (plan->prm.bucket == 0 && variant > decode_num_variants()) {
+        set_error("set_variant: decode kernel has %d variants", decode_num_variants());
+        return DET_ERR_INVALID_ARG;
+    }
+    plan->variant = variant;
+    return DET_OK;
+}
+
+struct GreenHandle {
+    CUgreenCtx gctx;
+    CUstream stream;
+};
+
+det_status_t det_test_green_stream_create(int sm_count, void** stream_out, void** handle_out, int* sm_granted)
+{
+    if (!stream_out || !handle_out || sm_count < 1) { set_error("green: bad argument"); return DET_ERR_INVALID_ARG; }
+    typedef CUresult (*GetResFn)(CUdevice, CUdevResource*, CUdevResourceType);
+    typedef CUresult (*SplitFn)(CUdevResource*, unsigned int*, const CUdevResource*, CUdevResource*, unsigned int, unsigned int);
+    typedef CUresult (*GenDescFn)(CUdevResourceDesc*, CUdevResource*, unsigned int);
+    typedef CUresult (*CreateFn)(CUgreenCtx*, CUdevResourceDesc, CUdevice, unsigned int);
+    typedef CUresult (*StreamFn)(CUstream*, CUgreenCtx, unsigned int, int);
+    typedef CUresult (*DevGetFn)(CUdevice*, int);
+    static GetResFn get_res = driver_fn<GetResFn>("cuDeviceGetDevResource");
+    static SplitFn split = driver_fn<SplitFn>("cuDevSmResourceSplitByCount");
+    static GenDescFn gen_desc = driver_fn<GenDescFn>("cuDevResourceGenerateDesc");
+    static CreateFn create = driver_fn<CreateFn>("cuGreenCtxCreate");
+    static StreamFn stream_create = driver_fn<StreamFn>("cuGreenCtxStreamCreate");
+    static DevGetFn dev_get = driver_fn<DevGetFn>("cuDeviceGet");
+    if (!get_res || !split || !gen_desc || !create || !stream_create || !dev_get) {
+        set_error("green: the driver does not provide the green-context entry points");
+        return DET_ERR_CUDA;
+    }
+    int dev = 0;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce != cudaSuccess) return cuda_fail("green: cudaGetDevice", ce);
+    cudaFree(nullptr);   // make sure the primary context exists
+    CUdevice cudev;
+    CUresult r = dev_get(&cudev, dev);
+    CUdevResource all{}, part{}, rest{};
+    if (r == CUDA_SUCCESS) r = get_res(cudev, &all, CU_DEV_RESOURCE_TYPE_SM);
+    unsigned int groups = 1;
+    if (r == CUDA_SUCCESS) r = split(&part, &groups, &all, &rest, 0, (unsigned)sm_count);
+    CUdevResourceDesc desc{};
+    if (r == CUDA_SUCCESS) r = gen_desc(&desc, &part, 1);
+    GreenHandle* h = new (std::nothrow) GreenHandle();
+    if (!h) { set_error("green: host allocation failed"); return DET_ERR_ALLOC; }
+    if (r == CUDA_SUCCESS) r = create(&h->gctx, desc, cudev, CU_GREEN_CTX_DEFAULT_STREAM);
+    if (r == CUDA_SUCCESS) r = stream_create(&h->stream, h->gctx, CU_STREAM_NON_BLOCKING, 0);
+    if (r != CUDA_SUCCESS) {
+        set_error("green: driver refused (CUresult %d)", (int)r);
+        delete h;
+        return DET_ERR_CUDA;
+    }
+    if (sm_granted) *sm_granted = (int)part.sm.smCount;
+    *stream_out = h->stream;
+    *handle_out = h;
+    return DET_OK;
+}
+
+void det_test_green_stream_destroy(void* handle)
+{
+    if (!handle) return;
+    GreenHandle* h = static_cast<GreenHandle*>(handle);
+    typedef CUresult (*StreamDestroyFn)(CUstream);
+    typedef CUresult (*DestroyFn)(CUgreenCtx);
+    static StreamDestroyFn sd = driver_fn<StreamDestroyFn>("cuStreamDestroy");
+    static DestroyFn gd = driver_fn<DestroyFn>("cuGreenCtxDestroy");
+    if (sd) sd(h->stream);
+    if (gd) gd(h->gctx);
+    delete h;
+}
+
+}  // extern "C"

@@ -1,0 +1,42 @@
+// Device helpers shared by the kernels: the register upcast of Eq. 2, explicit IEEE FMA / add (rule
+// R1: never rely on the compiler's contraction), packed FP32x2 FMA, and the adjacent-first lane tree.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace detlin {
+
+// up(): BF16 bit pattern -> binary32 with the pattern in the high half (exact).
+__device__ __forceinline__ float up_bf16(uint16_t h) { return __uint_as_float(((uint32_t)h) << 16); }
+// A 32-bit word holding two BF16 values (little endian: element k in the low half, k+1 in the high).
+__device__ __forceinline__ float up_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float up_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// fma.rn.f32x2: two independent IEEE-754 binary32 fused multiply-adds (round to nearest even, no
+// flush to zero) in one instruction; each half behaves exactly like fma.rn.f32.
+__device__ __forceinline__ void ffma2(unsigned long long& acc, unsigned long long a, unsigned long long b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
+// Balanced tree over the 32 lanes of a warp, adjacent lanes first (xor 1, 2, 4, 8, 16 in that
+// order).  fadd is commutative, so both partners compute identical bits and every lane ends with
+// the tree's root.
+__device__ __forceinline__ float lane_tree_sum(float a)
+{
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) a = __fadd_rn(a, __shfl_xor_sync(0xffffffffu, a, d));
+    return a;
+}
+
+}  // namespace detlin

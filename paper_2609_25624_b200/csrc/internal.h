@@ -1,0 +1,78 @@
+// Internal declarations shared by the host-side translation units of libdet_linear.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <cstdint>
+#include <cstddef>
+#include "det_linear.h"
+
+namespace detlin {
+
+constexpr int kOrderVersion = 1;
+constexpr int kSegmentGranule = 256;   // segment boundaries are multiples of this many k elements
+constexpr int kDecodeMaxM = 64;        // decode bucket edge (rule R2: "decode-shaped GEMMs (M <= 64)")
+
+enum KernelId : int { kKernelGeneric = 0, kKernelDecode = 1, kKernelPrefill = 2 };
+
+// Device-side status word written by kernels that give up a bounded wait.
+struct DeviceStatus {
+    unsigned int timeout_flag;   // nonzero: some wait expired
+    unsigned int where;          // which wait (diagnostic)
+};
+
+void set_error(const char* fmt, ...);
+det_status_t fill_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* out);
+
+// ---- kernel launchers (defined in the .cu files) -------------------------------------------
+struct LaunchArgs {
+    const float* x;
+    const uint16_t* W;
+    const float* b;
+    float* y;             // final output [M,N]
+    float* partials;      // [S,M,N] when S > 1, else nullptr
+    int64_t M, N, K;
+    int64_t seg_len;
+    int S;
+    cudaStream_t stream;
+    DeviceStatus* status; // device pointer
+    int sm_count;
+    int max_blocks;       // 0 = automatic
+    int variant;          // 0 = automatic
+};
+
+cudaError_t launch_generic(const LaunchArgs& a, int bucket);
+// Second pass of split-K: y[m,n] = (((P0 + P1) + P2) + ...) (+ b[n]); rule R3.
+cudaError_t launch_combine(const LaunchArgs& a);
+cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x);
+cudaError_t launch_prefill(const LaunchArgs& a);
+cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cudaStream_t stream);
+
+// Decode-kernel tiling chosen for a shape (numerically inert); used by the host to build the
+// tensor maps with matching box sizes.
+struct DecodeConfig {
+    int mt, wm, rt, wr, kc, stages;   // warp tile (mt x rt), warps (wm x wr), k per stage, ring depth
+    int id;
+};
+bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfig* out);
+int decode_num_variants();
+
+}  // namespace detlin
+
+struct det_linear_plan {
+    det_linear_params_t prm;
+    int device;
+    int sm_count;
+    float* partials;                 // device, S*M*N floats or nullptr
+    detlin::DeviceStatus* status;    // device
+    float* x_stage;                  // device staging for det_linear_run_host
+    float* y_stage;
+    int forced_kernel;               // -1 automatic
+    int max_blocks;
+    int variant;
+    // tensor-map cache for the decode kernel (keyed by the pointers they were built for)
+    const void* map_w_ptr;
+    const void* map_x_ptr;
+    int map_cfg_id;
+    CUtensorMap map_w;
+    CUtensorMap map_x;
+};

@@ -1,0 +1,385 @@
+// Decode kernel (bucket M <= 64): streams BF16 weight tiles from HBM through a TMA -> shared-memory
+// ring, widens them to FP32 in registers (Eq. 2) and accumulates with packed IEEE FP32 FMAs
+// (fma.rn.f32x2; rule R1) in the frozen decode order (V=4, L=32, P=2):
+//
+//   lane l of a warp owns k = c + 4l + j (j = 0..3) of every 128-element chunk c; its even
+//   elements feed sub-chain 0 and its odd elements sub-chain 1, which are exactly the two halves
+//   of one FP32x2 accumulator; the 64 leaves of an output are then summed adjacent-first
+//   (sub-chains inside the lane, then lanes xor 1, 2, 4, 8, 16).
+//
+// Everything else is schedule and therefore numerically inert (supplement C on rule R2: tile
+// sizes, warp counts and pipeline depth do not change the reduction tree): one producer warp
+// issues the bulk-tensor copies, WM x WR consumer warps each own an (MT batch rows) x (RT weight
+// rows) register tile, thread blocks walk (row tile, segment, batch block) work units in a strided
+// loop.  Rule R4 holds by construction: nothing that touches the order reads M.
+//
+// Every wait on a completion barrier is bounded; a wait that expires records the fact in the
+// plan's device status word and the block drains and returns.
+#include "internal.h"
+#include "device_utils.cuh"
+
+namespace detlin {
+
+namespace {
+
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false if the block is aborting or the wait expired (then it marks the
+// block as aborting and records the site in the device status word).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
+                                           unsigned site)
+{
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicExch(&status->where, site);
+            atomicExch(&status->timeout_flag, 1u);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
+                                          unsigned site)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status, site);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                            unsigned long long policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
+        : "memory");
+}
+
+template <int MT, int WM, int RT, int WR, int KC, int STAGES>
+struct Cfg {
+    static constexpr int kConsumerWarps = WM * WR;
+    static constexpr int kThreads = (kConsumerWarps + 1) * 32;
+    static constexpr int kMB = MT * WM;                       // batch rows per x box
+    static constexpr int kRB = RT * WR;                       // weight rows per block tile
+    static constexpr int kXBytes = kMB * KC * 4;
+    static constexpr int kWBoxBytes = RT * KC * 2;
+    static constexpr int kStageBytes = kXBytes + WR * kWBoxBytes;
+    static constexpr int kBarBytes = 128;                     // 2*STAGES barriers + abort flag
+    static constexpr int kSmemBytes = STAGES * kStageBytes + kBarBytes + 128;   // +128 for alignment
+    static_assert(STAGES >= 2 && STAGES <= 7, "ring depth");
+    static_assert(KC % 128 == 0 && KC <= 256, "a stage holds whole 128-element chunks; TMA boxes are <= 256 wide");
+    static_assert(kXBytes % 128 == 0 && kWBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
+};
+
+// Butterfly reduce-scatter over the 32 lanes that realises the adjacent-first tree: at step i
+// lanes l and l ^ (1 << i) exchange halves of their value arrays and add, so each lane ends with
+// NV/32 (at least 1) tree roots.  Lane with bit i set keeps the upper half at step i.
+template <int NV>
+__device__ __forceinline__ void lane_tree_scatter(float (&v)[NV], int lane)
+{
+    int n = NV;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        const int d = 1 << i;
+        if (n > 1) {
+            const int half = n >> 1;
+            const bool hi = (lane >> i) & 1;
+#pragma unroll
+            for (int t = 0; t < NV / 2; ++t) {
+                if (t < half) {
+                    const float send = hi ? v[t] : v[t + half];
+                    const float keep = hi ? v[t + half] : v[t];
+                    v[t] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, d));
+                }
+            }
+            n = half;
+        } else {
+            v[0] = __fadd_rn(v[0], __shfl_xor_sync(0xffffffffu, v[0], d));
+        }
+    }
+}
+
+template <int MT, int WM, int RT, int WR, int KC, int STAGES>
+__global__ void __launch_bounds__((WM * WR + 1) * 32, 1)
+decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+              const float* __restrict__ bias, float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct,
+              int n_row_tiles, int n_mblocks, DeviceStatus* status)
+{
+    using C = Cfg<MT, WM, RT, WR, KC, STAGES>;
+    extern __shared__ unsigned char smem_raw[];
+    // 128-byte aligned base (TMA destination requirement)
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    unsigned char* bar_mem = smem + STAGES * C::kStageBytes;
+    const uint32_t full0 = smem_u32(bar_mem);                 // full[s]  at full0 + 8 s
+    const uint32_t empty0 = full0 + 8 * STAGES;               // empty[s] at empty0 + 8 s
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 16 * STAGES);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, C::kConsumerWarps);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const long long total_units = (long long)n_row_tiles * S * n_mblocks;
+
+    if (warp == C::kConsumerWarps) {
+        // ---------------- producer warp: one lane issues all bulk-tensor copies ----------------
+        if (lane == 0) {
+            unsigned long long pol_w, pol_x;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_w));
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_x));
+            unsigned it = 0;
+            bool ok = true;
+            for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
+                const int tile = (int)(u % n_row_tiles);
+                const long long r = u / n_row_tiles;
+                const int s = (int)(r % S);
+                const int mb = (int)(r / S);
+                const int k_lo = s * seg_len;
+                const int k_hi = min(K, k_lo + seg_len);
+                const int n0 = tile * C::kRB;
+                for (int k0 = k_lo; k0 < k_hi; k0 += KC, ++it) {
+                    const int st = it % STAGES;
+                    const unsigned use = it / STAGES;
+                    if (use > 0 && !mbar_wait(empty0 + 8 * st, (use - 1) & 1, abort_flag, status, 1)) { ok = false; break; }
+                    const uint32_t fb = full0 + 8 * st;
+                    mbar_arrive_expect_tx(fb, C::kStageBytes);
+                    const uint32_t sbase = smem_u32(smem + st * C::kStageBytes);
+                    tma_load_2d(sbase, &map_x, k0, mb * C::kMB, fb, pol_x);
+#pragma unroll
+                    for (int wr = 0; wr < WR; ++wr)
+                        tma_load_2d(sbase + C::kXBytes + wr * C::kWBoxBytes, &map_w, k0, n0 + wr * RT, fb, pol_w);
+                }
+            }
+            if (!ok) {
+                // aborting: wait (bounded) for the copies this thread still has in flight
+                const unsigned first = it > (unsigned)STAGES ? it - STAGES : 0u;
+                for (unsigned j = first; j < it; ++j) {
+                    const unsigned long long t0 = global_timer_ns();
+                    while (!mbar_try_wait(full0 + 8 * (j % STAGES), (j / STAGES) & 1))
+                        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+                }
+            }
+        }
+    } else {
+        // ---------------- consumer warps ----------------
+        const int wm = warp % WM;
+        const int wr = warp / WM;
+        unsigned it = 0;
+        bool ok = true;
+        for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
+            const int tile = (int)(u % n_row_tiles);
+            const long long r = u / n_row_tiles;
+            const int s = (int)(r % S);
+            const int mb = (int)(r / S);
+            const int k_lo = s * seg_len;
+            const int k_hi = min(K, k_lo + seg_len);
+
+            unsigned long long acc[MT][RT];
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+#pragma unroll
+                for (int q = 0; q < RT; ++q) acc[m][q] = 0ull;   // (+0.0f, +0.0f)
+
+            for (int k0 = k_lo; k0 < k_hi; k0 += KC, ++it) {
+                const int st = it % STAGES;
+                if (!mbar_wait(full0 + 8 * st, (it / STAGES) & 1, abort_flag, status, 2)) { ok = false; break; }
+                const unsigned char* xs = smem + st * C::kStageBytes + (wm * MT) * (KC * 4) + lane * 16;
+                const unsigned char* ws = smem + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * 8;
+#pragma unroll
+                for (int cc = 0; cc < KC / 128; ++cc) {
+                    // elements beyond the end of K are skipped, not zero-filled (K % 4 == 0 here, so a
+                    // lane's four elements are all inside or all outside)
+                    if (k0 + cc * 128 + 4 * lane < k_hi) {
+                        unsigned long long wp[RT][2];
+#pragma unroll
+                        for (int q = 0; q < RT; ++q) {
+                            const uint2 w = *reinterpret_cast<const uint2*>(ws + q * (KC * 2) + cc * 256);
+                            wp[q][0] = pack2(up_lo(w.x), up_hi(w.x));
+                            wp[q][1] = pack2(up_lo(w.y), up_hi(w.y));
+                        }
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) {
+                            const ulonglong2 xv = *reinterpret_cast<const ulonglong2*>(xs + m * (KC * 4) + cc * 512);
+#pragma unroll
+                            for (int q = 0; q < RT; ++q) {
+                                ffma2(acc[m][q], xv.x, wp[q][0]);
+                                ffma2(acc[m][q], xv.y, wp[q][1]);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * st);
+            }
+            if (!ok) break;
+
+            // ---- epilogue: sub-chains, lane tree, bias, store ----
+            float v[MT * RT];
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+#pragma unroll
+                for (int q = 0; q < RT; ++q) {
+                    float e, o;
+                    unpack2(acc[m][q], e, o);
+                    v[m * RT + q] = __fadd_rn(e, o);
+                }
+            lane_tree_scatter<MT * RT>(v, lane);
+            constexpr int NV = MT * RT;
+            constexpr int kKeep = NV >= 32 ? NV / 32 : 1;
+            // index of v[0] in the (m, q) tile: bit i of the lane selected the upper half at step i
+            int base = 0;
+            {
+                int n = NV;
+#pragma unroll
+                for (int i = 0; i < 5; ++i)
+                    if (n > 1) { n >>= 1; base += ((lane >> i) & 1) * n; }
+            }
+            // with fewer than 32 values the lanes that differ only in their high bits hold the same root;
+            // the one whose high bits are zero stores it
+            constexpr int kLog2NV = NV >= 32 ? 5 : NV == 16 ? 4 : NV == 8 ? 3 : NV == 4 ? 2 : NV == 2 ? 1 : 0;
+            const bool owner = (lane >> kLog2NV) == 0;
+            if (owner) {
+#pragma unroll
+                for (int t = 0; t < kKeep; ++t) {
+                    const int idx = base + t;
+                    const int m = mb * C::kMB + wm * MT + idx / RT;
+                    const int n = tile * C::kRB + wr * RT + idx % RT;
+                    if (m < M && n < N) {
+                        float r0 = v[t];
+                        if (direct) {
+                            if (bias) r0 = __fadd_rn(r0, bias[n]);
+                            out[(long long)m * N + n] = r0;
+                        } else {
+                            out[((long long)s * M + m) * N + n] = r0;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+}
+
+typedef cudaError_t (*DecodeLaunchFn)(const LaunchArgs&, const CUtensorMap*, const CUtensorMap*);
+
+template <int MT, int WM, int RT, int WR, int KC, int STAGES>
+cudaError_t launch_decode_t(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
+{
+    using C = Cfg<MT, WM, RT, WR, KC, STAGES>;
+    auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES>;
+    static int blocks_per_sm = 0;
+    if (blocks_per_sm == 0) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        int occ = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, C::kThreads, C::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        blocks_per_sm = occ > 0 ? occ : 1;
+    }
+    const int n_row_tiles = (int)((a.N + C::kRB - 1) / C::kRB);
+    const int n_mblocks = (int)((a.M + C::kMB - 1) / C::kMB);
+    const long long units = (long long)n_row_tiles * a.S * n_mblocks;
+    long long grid = (long long)a.sm_count * blocks_per_sm;
+    if (a.max_blocks > 0 && grid > a.max_blocks) grid = a.max_blocks;
+    if (grid > units) grid = units;
+    const int direct = (a.S == 1);
+    kern<<<(unsigned)grid, C::kThreads, C::kSmemBytes, a.stream>>>(*map_w, *map_x, a.b, direct ? a.y : a.partials, (int)a.M,
+                                                                   (int)a.N, (int)a.K, (int)a.seg_len, a.S, direct,
+                                                                   n_row_tiles, n_mblocks, a.status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (!direct) return launch_combine(a);
+    return cudaSuccess;
+}
+
+struct DecodeEntry {
+    DecodeConfig cfg;
+    DecodeLaunchFn fn;
+};
+
+#define DEC(MT, WM, RT, WR, KC, ST) \
+    { {MT, WM, RT, WR, KC, ST, 0}, &launch_decode_t<MT, WM, RT, WR, KC, ST> }
+
+// Tilings per batch class (all produce identical bits).  The first entry of a class is the
+// automatic choice unless decode_pick() says otherwise.
+constexpr int kVariantsPerClass = 4;
+const DecodeEntry kTable[6][kVariantsPerClass] = {
+    /* M <= 1  */ {DEC(1, 1, 8, 2, 256, 6), DEC(1, 1, 8, 4, 256, 4), DEC(1, 1, 4, 4, 256, 6), DEC(1, 1, 16, 2, 256, 4)},
+    /* M <= 2  */ {DEC(2, 1, 8, 2, 256, 6), DEC(2, 1, 8, 4, 256, 4), DEC(2, 1, 4, 4, 256, 6), DEC(2, 1, 16, 2, 256, 4)},
+    /* M <= 4  */ {DEC(4, 1, 8, 2, 256, 6), DEC(4, 1, 8, 4, 256, 4), DEC(4, 1, 4, 4, 256, 6), DEC(4, 1, 4, 8, 128, 6)},
+    /* M <= 8  */ {DEC(8, 1, 8, 2, 128, 6), DEC(8, 1, 8, 4, 128, 4), DEC(8, 1, 4, 4, 128, 6), DEC(8, 1, 4, 8, 128, 4)},
+    /* M <= 16 */ {DEC(8, 2, 8, 2, 128, 4), DEC(8, 2, 4, 4, 128, 4), DEC(8, 2, 8, 1, 128, 6), DEC(8, 2, 4, 2, 128, 6)},
+    /* M > 16  */ {DEC(8, 4, 8, 1, 128, 4), DEC(8, 4, 4, 2, 128, 6), DEC(8, 4, 4, 1, 128, 6), DEC(8, 4, 8, 1, 128, 6)},
+};
+
+int m_class(int64_t M) { return M <= 1 ? 0 : M <= 2 ? 1 : M <= 4 ? 2 : M <= 8 ? 3 : M <= 16 ? 4 : 5; }
+
+}  // namespace
+
+int decode_num_variants() { return kVariantsPerClass; }
+
+bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfig* out)
+{
+    (void)N; (void)K;
+    if (variant < 0 || variant > kVariantsPerClass) return false;
+    const int cls = m_class(M);
+    const int v = variant == 0 ? 0 : variant - 1;
+    *out = kTable[cls][v].cfg;
+    out->id = cls * kVariantsPerClass + v;
+    return true;
+}
+
+cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
+{
+    DecodeConfig cfg;
+    if (!decode_config_for(a.M, a.N, a.K, a.variant, &cfg)) return cudaErrorInvalidValue;
+    return kTable[cfg.id / kVariantsPerClass][cfg.id % kVariantsPerClass].fn(a, map_w, map_x);
+}
+
+}  // namespace detlin

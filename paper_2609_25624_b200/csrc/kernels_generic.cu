@@ -1,0 +1,171 @@
+// Generic kernels: any shape, any alignment, scalar bounds-checked loads.  They execute exactly the
+// frozen order and serve ragged shapes (K % 8 != 0, misaligned buffers: the "masked code paths" of
+// the paper's ragged probe), the split-K second pass and the row argmax.  They are not tuned.
+#include "internal.h"
+#include "device_utils.cuh"
+
+namespace detlin {
+
+// Decode order (V=4, L=32, P=2): one warp per (row n, segment s); lane l owns k = c + 4l + j in every
+// 128-element chunk and feeds sub-chain j & 1; leaves are summed adjacent-first.
+__global__ void __launch_bounds__(256)
+generic_decode_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, const float* __restrict__ b,
+                      float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (warp >= N * S) return;
+    const int64_t n = warp / S;
+    const int s = (int)(warp % S);
+    const int64_t k_lo = (int64_t)s * seg_len;
+    const int64_t k_hi = (k_lo + seg_len < K) ? k_lo + seg_len : K;
+    const uint16_t* wrow = W + n * K;
+    for (int64_t m = 0; m < M; ++m) {
+        const float* xrow = x + m * K;
+        float a0 = 0.0f, a1 = 0.0f;
+        for (int64_t c = k_lo; c < k_hi; c += 128) {
+            const int64_t k0 = c + 4 * lane;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t k = k0 + j;
+                if (k < k_hi) {
+                    const float xv = xrow[k];
+                    const float wv = up_bf16(wrow[k]);
+                    if (j & 1) a1 = __fmaf_rn(xv, wv, a1);
+                    else       a0 = __fmaf_rn(xv, wv, a0);
+                }
+            }
+        }
+        float t = lane_tree_sum(__fadd_rn(a0, a1));
+        if (lane == 0) {
+            if (direct) out[m * N + n] = b ? __fadd_rn(t, b[n]) : t;
+            else        out[((int64_t)s * M + m) * N + n] = t;
+        }
+    }
+}
+
+// Prefill order (V=2, L=1, P=2): one thread per (m, n, segment): an even-k chain and an odd-k chain,
+// added once at the end of the segment.
+__global__ void __launch_bounds__(256)
+generic_prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, const float* __restrict__ b,
+                       float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct)
+{
+    const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t m = blockIdx.y;
+    const int s = blockIdx.z;
+    if (n >= N) return;
+    const int64_t k_lo = (int64_t)s * seg_len;
+    const int64_t k_hi = (k_lo + seg_len < K) ? k_lo + seg_len : K;
+    const float* xrow = x + m * K;
+    const uint16_t* wrow = W + n * K;
+    float a0 = 0.0f, a1 = 0.0f;
+    for (int64_t k = k_lo; k < k_hi; k += 2) {
+        a0 = __fmaf_rn(xrow[k], up_bf16(wrow[k]), a0);
+        if (k + 1 < k_hi) a1 = __fmaf_rn(xrow[k + 1], up_bf16(wrow[k + 1]), a1);
+    }
+    const float t = __fadd_rn(a0, a1);
+    if (direct) out[m * N + n] = b ? __fadd_rn(t, b[n]) : t;
+    else        out[((int64_t)s * M + m) * N + n] = t;
+}
+
+// Split-K second pass (rule R3): the S partials of every output are added in ascending segment
+// order by one thread, then the bias; no atomics anywhere.
+__global__ void __launch_bounds__(256)
+combine_kernel(const float* __restrict__ partials, const float* __restrict__ b, float* __restrict__ y,
+               int64_t MN, int64_t N, int S)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= MN) return;
+    float t = partials[i];
+    for (int s = 1; s < S; ++s) t = __fadd_rn(t, partials[(int64_t)s * MN + i]);
+    y[i] = b ? __fadd_rn(t, b[i % N]) : t;
+}
+
+cudaError_t launch_generic(const LaunchArgs& a, int bucket)
+{
+    const int direct = (a.S == 1);
+    float* out = direct ? a.y : a.partials;
+    if (bucket == 0) {
+        const int64_t warps = a.N * a.S;
+        const int64_t blocks = (warps + 7) / 8;
+        generic_decode_kernel<<<(unsigned)blocks, 256, 0, a.stream>>>(a.x, a.W, a.b, out, a.M, a.N, a.K,
+                                                                      a.seg_len, a.S, direct);
+    } else {
+        // grid.y carries M (< 65536 per launch); larger M is cut into slabs of rows
+        const int64_t max_y = 32768;
+        for (int64_t m0 = 0; m0 < a.M; m0 += max_y) {
+            const int64_t mm = (a.M - m0 < max_y) ? a.M - m0 : max_y;
+            dim3 grid((unsigned)((a.N + 255) / 256), (unsigned)mm, (unsigned)a.S);
+            float* o = out + m0 * a.N;   // both layouts ([M][N] and [s][M][N]) advance by whole rows
+            generic_prefill_kernel<<<grid, 256, 0, a.stream>>>(a.x + m0 * a.K, a.W, a.b, o, a.M, a.N, a.K,
+                                                              a.seg_len, a.S, direct);
+        }
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (!direct) return launch_combine(a);
+    return cudaSuccess;
+}
+
+cudaError_t launch_combine(const LaunchArgs& a)
+{
+    const int64_t MN = a.M * a.N;
+    combine_kernel<<<(unsigned)((MN + 255) / 256), 256, 0, a.stream>>>(a.partials, a.b, a.y, MN, a.N, a.S);
+    return cudaGetLastError();
+}
+
+// Row argmax, lowest index on ties (the paper's stated tie rule for greedy decoding).  One block
+// per row.  Ordering key: NaN beats everything (first NaN wins), otherwise larger value, then
+// smaller index.  Comparisons only, so the result is exact and order-free.
+__device__ __forceinline__ bool argmax_better(float v, int i, float bv, int bi)
+{
+    const bool vn = (v != v), bn = (bv != bv);
+    if (vn || bn) return vn && (!bn || i < bi);
+    return (v > bv) || (v == bv && i < bi);
+}
+
+__global__ void __launch_bounds__(1024)
+argmax_rows_kernel(const float* __restrict__ y, int64_t N, int32_t* __restrict__ idx)
+{
+    __shared__ float sv[32];
+    __shared__ int si[32];
+    const float* row = y + (int64_t)blockIdx.x * N;
+    float bv = row[0];
+    int bi = 0;
+    for (int64_t n = threadIdx.x; n < N; n += blockDim.x) {
+        const float v = row[n];
+        if (argmax_better(v, (int)n, bv, bi)) { bv = v; bi = (int)n; }
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
+        if (argmax_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int nw = blockDim.x >> 5;
+        bv = (threadIdx.x < nw) ? sv[threadIdx.x] : sv[0];
+        bi = (threadIdx.x < nw) ? si[threadIdx.x] : si[0];
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
+            if (argmax_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+        }
+        if (threadIdx.x == 0) idx[blockIdx.x] = bi;
+    }
+}
+
+cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cudaStream_t stream)
+{
+    const int64_t max_rows = 65535;
+    for (int64_t m0 = 0; m0 < M; m0 += max_rows) {
+        const int64_t mm = (M - m0 < max_rows) ? M - m0 : max_rows;
+        argmax_rows_kernel<<<(unsigned)mm, 1024, 0, stream>>>(y + m0 * N, N, idx + m0);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace detlin

@@ -1,0 +1,172 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle: bit-exact, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2609_25624_b200 import binding as B
+from paper_2609_25624_b200 import inputs
+from tests.gpu_util import (KERNEL_DECODE, KERNEL_GENERIC, KERNEL_PREFILL, assert_bits_equal, oracle_y,
+                            run_gpu)
+
+pytestmark = pytest.mark.gpu
+
+DECODE_SHAPES = [(1, 1024, 512), (1, 100, 512), (2, 77, 1000), (3, 130, 2304), (4, 96, 4096), (5, 33, 1024),
+                 (8, 257, 1536), (8, 64, 14336), (13, 200, 1000), (16, 96, 2048), (17, 40, 768), (32, 128, 4096),
+                 (33, 64, 640), (64, 50, 512), (7, 9, 8), (1, 1, 8), (64, 1, 256)]
+RAGGED_DECODE = [(1, 10, 1), (3, 17, 7), (5, 33, 1001), (8, 50, 1004), (4, 31, 250)]
+PREFILL_SHAPES = [(65, 129, 1000), (100, 1000, 1000), (130, 200, 1792), (128, 256, 1024), (200, 72, 4096),
+                  (65, 1, 8), (67, 5, 3)]
+
+
+def test_plan_params_match_oracle_rule():
+    for shp in DECODE_SHAPES + RAGGED_DECODE + PREFILL_SHAPES + [(8, 4096, 14336), (2048, 28672, 4096)]:
+        assert B.det_linear_plan_params(*shp).as_dict() == oracle.order_params(*shp), shp
+    plan = B.det_linear_plan(1, 1024, 512)
+    d = B.det_linear_plan_describe(plan)
+    assert (d["bucket"], d["V"], d["L"], d["P"], d["S"], d["seg_len"]) == ("decode", 4, 32, 2, 2, 256)
+    assert d["order_version"] == oracle.ORDER_VERSION == B.det_order_version()
+    plan.close()
+
+
+def test_config1_bit_exact():
+    """M=1, K=512, N=1024, seed 0, bias present: bit-exact against the oracle on every kernel."""
+    x, W, b = inputs.make_case(1, 1024, 512, seed=0)
+    want = oracle_y(x, W, b)
+    for kernel in (None, KERNEL_GENERIC, KERNEL_DECODE):
+        assert_bits_equal(run_gpu(x, W, b, kernel=kernel), want, f"kernel={kernel}")
+    assert_bits_equal(run_gpu(x, W, None), oracle_y(x, W, None), "no bias")
+
+
+@pytest.mark.parametrize("M,N,K", DECODE_SHAPES)
+def test_decode_bit_exact_all_tilings(M, N, K):
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    assert_bits_equal(run_gpu(x, W, b, kernel=KERNEL_GENERIC), want, "generic")
+    for variant in range(0, 5):
+        assert_bits_equal(run_gpu(x, W, b, kernel=KERNEL_DECODE, variant=variant), want, f"variant={variant}")
+    assert_bits_equal(run_gpu(x, W, b, max_blocks=1), want, "one block")
+    assert_bits_equal(run_gpu(x, W, b, max_blocks=3), want, "three blocks")
+
+
+@pytest.mark.parametrize("M,N,K", RAGGED_DECODE)
+def test_decode_ragged_bit_exact(M, N, K):
+    x, W, b = inputs.make_case(M, N, K)
+    assert_bits_equal(run_gpu(x, W, b), oracle_y(x, W, b), "ragged")
+
+
+@pytest.mark.parametrize("M,N,K", PREFILL_SHAPES)
+def test_prefill_bit_exact(M, N, K):
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    assert_bits_equal(run_gpu(x, W, b, kernel=KERNEL_GENERIC), want, "generic")
+    assert_bits_equal(run_gpu(x, W, b), want, "automatic")
+    assert_bits_equal(run_gpu(x, W, None), oracle_y(x, W, None), "no bias")
+
+
+def test_misaligned_buffers_take_generic_path_same_bits():
+    M, N, K = 4, 64, 512
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    xd = torch.empty(M * K + 1, dtype=torch.float32, device="cuda")[1:].view(M, K)
+    xd.copy_(x)
+    assert xd.data_ptr() % 16 != 0
+    y = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    plan = B.det_linear_plan(M, N, K)
+    B.det_linear_run(plan, xd, W.cuda(), b.cuda(), y)
+    B.det_linear_plan_check(plan)
+    assert_bits_equal(y.cpu().numpy(), want, "misaligned x")
+    plan.close()
+
+
+def test_special_values_bit_exact():
+    """Subnormals, signed zeros, large magnitudes and cancellations: gradual underflow and signed
+    zeros must match the oracle exactly (rule R1: IEEE-754 arithmetic, no flush to zero)."""
+    M, N, K = 8, 64, 1024
+    g = torch.Generator().manual_seed(99)
+    x = torch.randn(M, K, generator=g)
+    xb = x.view(torch.int32)
+    xb[0, :] = torch.randint(1, 1 << 23, (K,), generator=g, dtype=torch.int32)            # subnormals
+    xb[1, ::2] = torch.randint(1, 1 << 23, (K // 2,), generator=g, dtype=torch.int32) | (1 << 31)
+    x[2, :] = 0.0
+    x[3, :] = -0.0
+    x[4, :] *= 1e30
+    x[5, :] *= 1e-30
+    x[6, 1::2] = -x[6, ::2]
+    W = (0.02 * torch.randn(N, K, generator=g)).to(torch.bfloat16)
+    Wb = inputs.bf16_bits(W).copy()
+    Wb[0, :] = 0x0001                       # BF16 subnormal
+    Wb[1, :] = 0x8000                       # -0
+    Wb[2, :] = 0x7F7F                       # largest finite BF16
+    Wb[3, ::2] = Wb[3, 1::2]
+    W = inputs.bits_to_bf16(Wb)
+    x[4, :] = x[4, :].clamp(-1e30, 1e30)
+    want = oracle_y(x, W, None)
+    finite = np.isfinite(want)
+    for kernel in (KERNEL_GENERIC, KERNEL_DECODE):
+        got = run_gpu(x, W, None, kernel=kernel)
+        assert np.array_equal(np.isnan(got), np.isnan(want))
+        assert_bits_equal(np.where(np.isnan(want), 0, got), np.where(np.isnan(want), 0, want), f"kernel={kernel}")
+    assert finite.sum() > want.size // 2
+
+
+def test_batch_invariance_on_gpu():
+    """Rule R4: row m of a batch-M call equals the M = 1 call of that row, for M <= 64."""
+    N, K = 96, 2048
+    x, W, b = inputs.make_case(64, N, K, seed=3)
+    full = run_gpu(x, W, b)
+    assert_bits_equal(full, oracle_y(x, W, b), "M=64")
+    for M in (1, 2, 5, 8, 16, 31, 32, 33):
+        assert_bits_equal(run_gpu(x[:M].contiguous(), W, b), full[:M], f"M={M}")
+    assert_bits_equal(run_gpu(x[40:41].contiguous(), W, b), full[40:41], "row 40 alone")
+
+
+def test_argmax_rows_gpu():
+    g = torch.Generator().manual_seed(5)
+    y = torch.randn(9, 5000, generator=g)
+    y[2, 4000] = y[2, 17] = y[2].max() + 1
+    y[3, :] = 1.5
+    y[4, 0] = 100.0
+    y[5, 4999] = 100.0
+    y[6, 300] = float("nan")
+    y[7, 10] = 0.0
+    y[7, 11] = -0.0
+    y[7, :10] = -1
+    y[7, 12:] = -1
+    want = oracle.argmax_rows(y.numpy())
+    idx = torch.empty(9, dtype=torch.int32, device="cuda")
+    B.det_argmax_rows(y.cuda(), idx)
+    torch.cuda.synchronize()
+    assert idx.cpu().tolist() == want.tolist()
+    assert want[2] == 17 and want[3] == 0 and want[6] == 300 and want[7] == 10
+    # a single-column and a short row
+    for n in (1, 31, 1025):
+        z = torch.randn(3, n, generator=g)
+        idx = torch.empty(3, dtype=torch.int32, device="cuda")
+        B.det_argmax_rows(z.cuda(), idx)
+        assert idx.cpu().tolist() == oracle.argmax_rows(z.numpy()).tolist()
+
+
+def test_run_host_matches_device_run():
+    M, N, K = 8, 300, 1024
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    plan = B.det_linear_plan(M, N, K)
+    xh = x.pin_memory()
+    yh = torch.empty(M, N, dtype=torch.float32).pin_memory()
+    B.det_linear_run_host(plan, xh, W.cuda(), b.cuda(), yh)
+    assert_bits_equal(yh.numpy(), want, "run_host")
+    plan.close()
+
+
+def test_bad_arguments_are_rejected():
+    with pytest.raises(B.DetLinearError):
+        B.det_linear_plan(0, 4, 8)
+    with pytest.raises(B.DetLinearError):
+        B.det_linear_plan_params(1, -1, 8)
+    plan = B.det_linear_plan(2, 4, 8)
+    rc = B.lib().det_linear_run(plan.handle, None, None, None, None, None)
+    assert rc == 1 and "NULL" in B.det_last_error()
+    with pytest.raises(B.DetLinearError):
+        B.det_test_plan_force_kernel(plan, KERNEL_PREFILL)
+    plan.close()
