@@ -59,7 +59,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 
 // Bounded wait.  Returns false if the block is aborting or the wait expired (then it marks the
 // block as aborting and records the site in the device status word).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
                                            unsigned site)
 {
     const unsigned long long t0 = global_timer_ns();
@@ -92,18 +92,35 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
-template <int MT, int WM, int RT, int WR, int KC, int STAGES>
+// PG = warps in the producer group: 1 (plain) or 4 (a whole warpgroup, which lets the kernel move
+// registers from the producer to the consumers with setmaxnreg when the consumer tile is large).
+template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
 struct Cfg {
     static constexpr int kConsumerWarps = WM * WR;
-    static constexpr int kThreads = (kConsumerWarps + 1) * 32;
+    static constexpr int kThreads = (kConsumerWarps + PG) * 32;
     static constexpr int kMB = MT * WM;                       // batch rows per x box
     static constexpr int kRB = RT * WR;                       // weight rows per block tile
     static constexpr int kXBytes = kMB * KC * 4;
     static constexpr int kWBoxBytes = RT * KC * 2;
     static constexpr int kStageBytes = kXBytes + WR * kWBoxBytes;
-    static constexpr int kBarBytes = 128;                     // 2*STAGES barriers + abort flag
+    static constexpr int kBarBytes = 256;                     // 2*STAGES barriers + abort flag
     static constexpr int kSmemBytes = STAGES * kStageBytes + kBarBytes + 128;   // +128 for alignment
-    static_assert(STAGES >= 2 && STAGES <= 7, "ring depth");
+    // With a producer warpgroup the block is compiled for kMinBlocks blocks per SM and then moves
+    // registers inside its own allocation (threads x launch registers): producers shrink to
+    // kProducerRegs, consumers grow to kConsumerRegs.  setmaxnreg.inc blocks until the registers
+    // exist, so the request must never exceed what the block owns.
+    static constexpr int kMinBlocks = (PG == 4 && kConsumerWarps == 4) ? 2 : 1;
+    static constexpr int kLaunchRegsRaw = (65536 / (kMinBlocks * kThreads)) / 8 * 8;
+    static constexpr int kLaunchRegs = kLaunchRegsRaw > 255 ? 248 : kLaunchRegsRaw;
+    static constexpr int kProducerRegs = 32;
+    static constexpr int kConsumerRegsRaw =
+        PG == 4 ? ((kThreads * kLaunchRegs - PG * 32 * kProducerRegs) / (kConsumerWarps * 32)) / 8 * 8 : 0;
+    static constexpr int kConsumerRegs = kConsumerRegsRaw > 240 ? 240 : kConsumerRegsRaw;
+    static_assert(PG == 1 || kConsumerRegs * kConsumerWarps * 32 + kProducerRegs * PG * 32 <= kThreads * kLaunchRegs,
+                  "register move must fit in the block's own allocation");
+    static_assert(PG == 1 || kConsumerRegs >= kLaunchRegs, "consumers only ever grow");
+    static_assert(PG == 1 || (PG == 4 && kConsumerWarps % 4 == 0), "setmaxnreg works on whole warpgroups");
+    static_assert(STAGES >= 2 && STAGES <= 12, "ring depth");
     static_assert(KC % 128 == 0 && KC <= 256, "a stage holds whole 128-element chunks; TMA boxes are <= 256 wide");
     static_assert(kXBytes % 128 == 0 && kWBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
 };
@@ -136,13 +153,38 @@ __device__ __forceinline__ void lane_tree_scatter(float (&v)[NV], int lane)
     }
 }
 
-template <int MT, int WM, int RT, int WR, int KC, int STAGES>
-__global__ void __launch_bounds__((WM * WR + 1) * 32, 1)
+template <int REGS>
+__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS)); }
+template <int REGS>
+__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS)); }
+
+// Programmatic dependent launch: let the next kernel in the stream start its prologue early, and
+// wait for the previous kernel's results before touching anything it may have produced.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+struct Unit {
+    int tile, s, mb, k_lo, k_hi;
+};
+__device__ __forceinline__ Unit decode_unit(long long u, int n_row_tiles, int S, int seg_len, int K)
+{
+    Unit r;
+    r.tile = (int)(u % n_row_tiles);
+    const long long q = u / n_row_tiles;
+    r.s = (int)(q % S);
+    r.mb = (int)(q / S);
+    r.k_lo = r.s * seg_len;
+    r.k_hi = min(K, r.k_lo + seg_len);
+    return r;
+}
+
+template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
+__global__ void __launch_bounds__((WM * WR + PG) * 32, (Cfg<MT, WM, RT, WR, KC, STAGES, PG>::kMinBlocks))
 decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
               const float* __restrict__ bias, float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct,
               int n_row_tiles, int n_mblocks, DeviceStatus* status)
 {
-    using C = Cfg<MT, WM, RT, WR, KC, STAGES>;
+    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG>;
     extern __shared__ unsigned char smem_raw[];
     // 128-byte aligned base (TMA destination requirement)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -164,36 +206,56 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    pdl_launch_dependents();
 
     const long long total_units = (long long)n_row_tiles * S * n_mblocks;
 
-    if (warp == C::kConsumerWarps) {
-        // ---------------- producer warp: one lane issues all bulk-tensor copies ----------------
-        if (lane == 0) {
+    if (warp < PG) {
+        // ---------------- producer group: one lane issues all bulk-tensor copies ----------------
+        if (PG == 4) reg_dec<C::kProducerRegs>();
+        if (warp == 0 && lane == 0) {
             unsigned long long pol_w, pol_x;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_w));
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_x));
             unsigned it = 0;
             bool ok = true;
+            // Weights never depend on the previous kernel, activations may: the first ring of
+            // weight boxes is requested before waiting for the previous kernel to finish.
+            unsigned pre = 0;
+            {
+                long long u = blockIdx.x;
+                unsigned j = 0;
+                while (u < total_units && j < (unsigned)STAGES) {
+                    const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
+                    for (int k0 = un.k_lo; k0 < un.k_hi && j < (unsigned)STAGES; k0 += KC, ++j) {
+                        const uint32_t fb = full0 + 8 * j;
+                        mbar_arrive_expect_tx(fb, C::kStageBytes);
+                        const uint32_t sbase = smem_u32(smem + j * C::kStageBytes);
+#pragma unroll
+                        for (int wr = 0; wr < WR; ++wr)
+                            tma_load_2d(sbase + C::kXBytes + wr * C::kWBoxBytes, &map_w, k0, un.tile * C::kRB + wr * RT, fb, pol_w);
+                    }
+                    u += gridDim.x;
+                }
+                pre = j;
+            }
+            pdl_wait();
             for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
-                const int tile = (int)(u % n_row_tiles);
-                const long long r = u / n_row_tiles;
-                const int s = (int)(r % S);
-                const int mb = (int)(r / S);
-                const int k_lo = s * seg_len;
-                const int k_hi = min(K, k_lo + seg_len);
-                const int n0 = tile * C::kRB;
-                for (int k0 = k_lo; k0 < k_hi; k0 += KC, ++it) {
+                const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
+                const int n0 = un.tile * C::kRB;
+                for (int k0 = un.k_lo; k0 < un.k_hi; k0 += KC, ++it) {
                     const int st = it % STAGES;
                     const unsigned use = it / STAGES;
-                    if (use > 0 && !mbar_wait(empty0 + 8 * st, (use - 1) & 1, abort_flag, status, 1)) { ok = false; break; }
                     const uint32_t fb = full0 + 8 * st;
-                    mbar_arrive_expect_tx(fb, C::kStageBytes);
                     const uint32_t sbase = smem_u32(smem + st * C::kStageBytes);
-                    tma_load_2d(sbase, &map_x, k0, mb * C::kMB, fb, pol_x);
+                    if (it >= pre) {
+                        if (use > 0 && !mbar_wait(empty0 + 8 * st, (use - 1) & 1, abort_flag, status, 1)) { ok = false; break; }
+                        mbar_arrive_expect_tx(fb, C::kStageBytes);
 #pragma unroll
-                    for (int wr = 0; wr < WR; ++wr)
-                        tma_load_2d(sbase + C::kXBytes + wr * C::kWBoxBytes, &map_w, k0, n0 + wr * RT, fb, pol_w);
+                        for (int wr = 0; wr < WR; ++wr)
+                            tma_load_2d(sbase + C::kXBytes + wr * C::kWBoxBytes, &map_w, k0, n0 + wr * RT, fb, pol_w);
+                    }
+                    tma_load_2d(sbase, &map_x, k0, un.mb * C::kMB, fb, pol_x);
                 }
             }
             if (!ok) {
@@ -208,17 +270,15 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         }
     } else {
         // ---------------- consumer warps ----------------
-        const int wm = warp % WM;
-        const int wr = warp / WM;
+        if (PG == 4) reg_inc<C::kConsumerRegs>();
+        const int cw = warp - PG;
+        const int wm = cw % WM;
+        const int wr = cw / WM;
         unsigned it = 0;
         bool ok = true;
+        bool waited = false;
         for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
-            const int tile = (int)(u % n_row_tiles);
-            const long long r = u / n_row_tiles;
-            const int s = (int)(r % S);
-            const int mb = (int)(r / S);
-            const int k_lo = s * seg_len;
-            const int k_hi = min(K, k_lo + seg_len);
+            const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
 
             unsigned long long acc[MT][RT];
 #pragma unroll
@@ -226,16 +286,18 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
 #pragma unroll
                 for (int q = 0; q < RT; ++q) acc[m][q] = 0ull;   // (+0.0f, +0.0f)
 
-            for (int k0 = k_lo; k0 < k_hi; k0 += KC, ++it) {
+            for (int k0 = un.k_lo; k0 < un.k_hi; k0 += KC, ++it) {
                 const int st = it % STAGES;
                 if (!mbar_wait(full0 + 8 * st, (it / STAGES) & 1, abort_flag, status, 2)) { ok = false; break; }
                 const unsigned char* xs = smem + st * C::kStageBytes + (wm * MT) * (KC * 4) + lane * 16;
                 const unsigned char* ws = smem + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * 8;
-#pragma unroll
+#pragma unroll(MT * RT >= 64 ? 1 : 2)
                 for (int cc = 0; cc < KC / 128; ++cc) {
-                    // elements beyond the end of K are skipped, not zero-filled (K % 4 == 0 here, so a
-                    // lane's four elements are all inside or all outside)
-                    if (k0 + cc * 128 + 4 * lane < k_hi) {
+                    // Elements beyond the end of K are skipped, not zero-filled (K % 4 == 0 here, so a
+                    // lane's four elements are all inside or all outside).  Whole chunks take the
+                    // warp-uniform branch.
+                    const int kc0 = k0 + cc * 128;
+                    if (kc0 + 128 <= un.k_hi || kc0 + 4 * lane < un.k_hi) {
                         unsigned long long wp[RT][2];
 #pragma unroll
                         for (int q = 0; q < RT; ++q) {
@@ -247,10 +309,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                         for (int m = 0; m < MT; ++m) {
                             const ulonglong2 xv = *reinterpret_cast<const ulonglong2*>(xs + m * (KC * 4) + cc * 512);
 #pragma unroll
-                            for (int q = 0; q < RT; ++q) {
-                                ffma2(acc[m][q], xv.x, wp[q][0]);
-                                ffma2(acc[m][q], xv.y, wp[q][1]);
-                            }
+                            for (int q = 0; q < RT; ++q) ffma2(acc[m][q], xv.x, wp[q][0]);
+#pragma unroll
+                            for (int q = 0; q < RT; ++q) ffma2(acc[m][q], xv.y, wp[q][1]);
                         }
                     }
                 }
@@ -284,19 +345,21 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             // the one whose high bits are zero stores it
             constexpr int kLog2NV = NV >= 32 ? 5 : NV == 16 ? 4 : NV == 8 ? 3 : NV == 4 ? 2 : NV == 2 ? 1 : 0;
             const bool owner = (lane >> kLog2NV) == 0;
+            // the output buffer may still be read by the previous kernel in the stream
+            if (!waited) { pdl_wait(); waited = true; }
             if (owner) {
 #pragma unroll
                 for (int t = 0; t < kKeep; ++t) {
                     const int idx = base + t;
-                    const int m = mb * C::kMB + wm * MT + idx / RT;
-                    const int n = tile * C::kRB + wr * RT + idx % RT;
+                    const int m = un.mb * C::kMB + wm * MT + idx / RT;
+                    const int n = un.tile * C::kRB + wr * RT + idx % RT;
                     if (m < M && n < N) {
                         float r0 = v[t];
                         if (direct) {
                             if (bias) r0 = __fadd_rn(r0, bias[n]);
                             out[(long long)m * N + n] = r0;
                         } else {
-                            out[((long long)s * M + m) * N + n] = r0;
+                            out[((long long)un.s * M + m) * N + n] = r0;
                         }
                     }
                 }
@@ -308,11 +371,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
 
 typedef cudaError_t (*DecodeLaunchFn)(const LaunchArgs&, const CUtensorMap*, const CUtensorMap*);
 
-template <int MT, int WM, int RT, int WR, int KC, int STAGES>
+template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
 cudaError_t launch_decode_t(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
 {
-    using C = Cfg<MT, WM, RT, WR, KC, STAGES>;
-    auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES>;
+    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG>;
+    auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES, PG>;
     static int blocks_per_sm = 0;
     if (blocks_per_sm == 0) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
@@ -329,10 +392,19 @@ cudaError_t launch_decode_t(const LaunchArgs& a, const CUtensorMap* map_w, const
     if (a.max_blocks > 0 && grid > a.max_blocks) grid = a.max_blocks;
     if (grid > units) grid = units;
     const int direct = (a.S == 1);
-    kern<<<(unsigned)grid, C::kThreads, C::kSmemBytes, a.stream>>>(*map_w, *map_x, a.b, direct ? a.y : a.partials, (int)a.M,
-                                                                   (int)a.N, (int)a.K, (int)a.seg_len, a.S, direct,
-                                                                   n_row_tiles, n_mblocks, a.status);
-    cudaError_t e = cudaGetLastError();
+
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(C::kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, *map_w, *map_x, a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N,
+                                       (int)a.K, (int)a.seg_len, a.S, direct, n_row_tiles, n_mblocks, a.status);
     if (e != cudaSuccess) return e;
     if (!direct) return launch_combine(a);
     return cudaSuccess;
@@ -343,19 +415,19 @@ struct DecodeEntry {
     DecodeLaunchFn fn;
 };
 
-#define DEC(MT, WM, RT, WR, KC, ST) \
-    { {MT, WM, RT, WR, KC, ST, 0}, &launch_decode_t<MT, WM, RT, WR, KC, ST> }
+#define DEC(MT, WM, RT, WR, KC, ST, PG) \
+    { {MT, WM, RT, WR, KC, ST, 0}, &launch_decode_t<MT, WM, RT, WR, KC, ST, PG> }
 
 // Tilings per batch class (all produce identical bits).  The first entry of a class is the
-// automatic choice unless decode_pick() says otherwise.
+// automatic choice.
 constexpr int kVariantsPerClass = 4;
 const DecodeEntry kTable[6][kVariantsPerClass] = {
-    /* M <= 1  */ {DEC(1, 1, 8, 2, 256, 6), DEC(1, 1, 8, 4, 256, 4), DEC(1, 1, 4, 4, 256, 6), DEC(1, 1, 16, 2, 256, 4)},
-    /* M <= 2  */ {DEC(2, 1, 8, 2, 256, 6), DEC(2, 1, 8, 4, 256, 4), DEC(2, 1, 4, 4, 256, 6), DEC(2, 1, 16, 2, 256, 4)},
-    /* M <= 4  */ {DEC(4, 1, 8, 2, 256, 6), DEC(4, 1, 8, 4, 256, 4), DEC(4, 1, 4, 4, 256, 6), DEC(4, 1, 4, 8, 128, 6)},
-    /* M <= 8  */ {DEC(8, 1, 8, 2, 128, 6), DEC(8, 1, 8, 4, 128, 4), DEC(8, 1, 4, 4, 128, 6), DEC(8, 1, 4, 8, 128, 4)},
-    /* M <= 16 */ {DEC(8, 2, 8, 2, 128, 4), DEC(8, 2, 4, 4, 128, 4), DEC(8, 2, 8, 1, 128, 6), DEC(8, 2, 4, 2, 128, 6)},
-    /* M > 16  */ {DEC(8, 4, 8, 1, 128, 4), DEC(8, 4, 4, 2, 128, 6), DEC(8, 4, 4, 1, 128, 6), DEC(8, 4, 8, 1, 128, 6)},
+    /* M <= 1  */ {DEC(1, 1, 4, 4, 256, 8, 1), DEC(1, 1, 8, 4, 256, 6, 1), DEC(1, 1, 8, 2, 256, 6, 1), DEC(1, 1, 2, 4, 256, 8, 1)},
+    /* M <= 2  */ {DEC(2, 1, 4, 4, 256, 8, 1), DEC(2, 1, 8, 4, 256, 6, 1), DEC(2, 1, 8, 2, 256, 6, 1), DEC(2, 1, 2, 4, 256, 8, 1)},
+    /* M <= 4  */ {DEC(4, 1, 4, 4, 256, 6, 1), DEC(4, 1, 8, 4, 256, 4, 1), DEC(4, 1, 8, 2, 256, 6, 1), DEC(4, 1, 4, 8, 256, 4, 1)},
+    /* M <= 8  */ {DEC(8, 1, 4, 4, 256, 5, 1), DEC(8, 1, 8, 8, 256, 3, 4), DEC(8, 1, 8, 4, 256, 4, 4), DEC(8, 1, 4, 8, 256, 4, 1)},
+    /* M <= 16 */ {DEC(8, 2, 8, 4, 256, 3, 4), DEC(8, 2, 4, 4, 256, 4, 1), DEC(8, 2, 8, 2, 256, 4, 4), DEC(8, 2, 4, 2, 256, 4, 1)},
+    /* M > 16  */ {DEC(8, 4, 8, 2, 128, 5, 4), DEC(8, 4, 4, 2, 128, 6, 1), DEC(8, 4, 8, 1, 128, 6, 4), DEC(8, 4, 4, 1, 128, 6, 1)},
 };
 
 int m_class(int64_t M) { return M <= 1 ? 0 : M <= 2 ? 1 : M <= 4 ? 2 : M <= 8 ? 3 : M <= 16 ? 4 : 5; }
