@@ -18,15 +18,21 @@ __device__ __forceinline__ void ffma2(unsigned long long& acc, unsigned long lon
 {
     asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
 }
+// Two FP32 values as one 64-bit FP32x2 operand (low half = first element).  Written with integer
+// operations so that the compiler can place the halves straight into a register pair.
 __device__ __forceinline__ unsigned long long pack2(float lo, float hi)
 {
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
+    return ((unsigned long long)__float_as_uint(hi) << 32) | (unsigned long long)__float_as_uint(lo);
 }
 __device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi)
 {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    lo = __uint_as_float((unsigned int)v);
+    hi = __uint_as_float((unsigned int)(v >> 32));
+}
+// A 32-bit word holding BF16 elements (k, k+1) -> the FP32x2 operand (up(k), up(k+1)).
+__device__ __forceinline__ unsigned long long up_pair(uint32_t w)
+{
+    return ((unsigned long long)(w & 0xffff0000u) << 32) | (unsigned long long)(w << 16);
 }
 
 // Balanced tree over the 32 lanes of a warp, adjacent lanes first (xor 1, 2, 4, 8, 16 in that

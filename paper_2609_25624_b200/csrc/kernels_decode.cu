@@ -23,6 +23,7 @@ namespace detlin {
 namespace {
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+constexpr unsigned kTryWaitHintNs = 2000;                   // a waiting thread may sleep this long per try
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -43,12 +44,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kTryWaitHintNs)
         : "memory");
     return ok != 0;
+}
+__device__ __forceinline__ float4 lds128(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ unsigned long long global_timer_ns()
 {
@@ -188,6 +201,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     extern __shared__ unsigned char smem_raw[];
     // 128-byte aligned base (TMA destination requirement)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    const uint32_t smem_base = smem_u32(smem);
     unsigned char* bar_mem = smem + STAGES * C::kStageBytes;
     const uint32_t full0 = smem_u32(bar_mem);                 // full[s]  at full0 + 8 s
     const uint32_t empty0 = full0 + 8 * STAGES;               // empty[s] at empty0 + 8 s
@@ -280,17 +294,17 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
             const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
 
-            unsigned long long acc[MT][RT];
+            float2 acc[MT][RT];          // (even-k sub-chain, odd-k sub-chain) of the lane's leaf pair
 #pragma unroll
             for (int m = 0; m < MT; ++m)
 #pragma unroll
-                for (int q = 0; q < RT; ++q) acc[m][q] = 0ull;   // (+0.0f, +0.0f)
+                for (int q = 0; q < RT; ++q) acc[m][q] = make_float2(0.0f, 0.0f);
 
             for (int k0 = un.k_lo; k0 < un.k_hi; k0 += KC, ++it) {
                 const int st = it % STAGES;
                 if (!mbar_wait(full0 + 8 * st, (it / STAGES) & 1, abort_flag, status, 2)) { ok = false; break; }
-                const unsigned char* xs = smem + st * C::kStageBytes + (wm * MT) * (KC * 4) + lane * 16;
-                const unsigned char* ws = smem + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * 8;
+                const uint32_t xs = smem_base + st * C::kStageBytes + (wm * MT) * (KC * 4) + lane * 16;
+                const uint32_t ws = smem_base + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * 8;
 #pragma unroll(MT * RT >= 64 ? 1 : 2)
                 for (int cc = 0; cc < KC / 128; ++cc) {
                     // Elements beyond the end of K are skipped, not zero-filled (K % 4 == 0 here, so a
@@ -298,20 +312,21 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                     // warp-uniform branch.
                     const int kc0 = k0 + cc * 128;
                     if (kc0 + 128 <= un.k_hi || kc0 + 4 * lane < un.k_hi) {
-                        unsigned long long wp[RT][2];
+                        float2 wp[RT][2];
 #pragma unroll
                         for (int q = 0; q < RT; ++q) {
-                            const uint2 w = *reinterpret_cast<const uint2*>(ws + q * (KC * 2) + cc * 256);
-                            wp[q][0] = pack2(up_lo(w.x), up_hi(w.x));
-                            wp[q][1] = pack2(up_lo(w.y), up_hi(w.y));
+                            const uint2 w = lds64(ws + q * (KC * 2) + cc * 256);
+                            wp[q][0] = make_float2(up_lo(w.x), up_hi(w.x));
+                            wp[q][1] = make_float2(up_lo(w.y), up_hi(w.y));
                         }
 #pragma unroll
                         for (int m = 0; m < MT; ++m) {
-                            const ulonglong2 xv = *reinterpret_cast<const ulonglong2*>(xs + m * (KC * 4) + cc * 512);
+                            const float4 xv = lds128(xs + m * (KC * 4) + cc * 512);
+                            const float2 x01 = make_float2(xv.x, xv.y), x23 = make_float2(xv.z, xv.w);
 #pragma unroll
-                            for (int q = 0; q < RT; ++q) ffma2(acc[m][q], xv.x, wp[q][0]);
+                            for (int q = 0; q < RT; ++q) acc[m][q] = __ffma2_rn(x01, wp[q][0], acc[m][q]);
 #pragma unroll
-                            for (int q = 0; q < RT; ++q) ffma2(acc[m][q], xv.y, wp[q][1]);
+                            for (int q = 0; q < RT; ++q) acc[m][q] = __ffma2_rn(x23, wp[q][1], acc[m][q]);
                         }
                     }
                 }
@@ -325,11 +340,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
 #pragma unroll
             for (int m = 0; m < MT; ++m)
 #pragma unroll
-                for (int q = 0; q < RT; ++q) {
-                    float e, o;
-                    unpack2(acc[m][q], e, o);
-                    v[m * RT + q] = __fadd_rn(e, o);
-                }
+                for (int q = 0; q < RT; ++q) v[m * RT + q] = __fadd_rn(acc[m][q].x, acc[m][q].y);
             lane_tree_scatter<MT * RT>(v, lane);
             constexpr int NV = MT * RT;
             constexpr int kKeep = NV >= 32 ? NV / 32 : 1;
@@ -425,9 +436,9 @@ const DecodeEntry kTable[6][kVariantsPerClass] = {
     /* M <= 1  */ {DEC(1, 1, 4, 4, 256, 8, 1), DEC(1, 1, 8, 4, 256, 6, 1), DEC(1, 1, 8, 2, 256, 6, 1), DEC(1, 1, 2, 4, 256, 8, 1)},
     /* M <= 2  */ {DEC(2, 1, 4, 4, 256, 8, 1), DEC(2, 1, 8, 4, 256, 6, 1), DEC(2, 1, 8, 2, 256, 6, 1), DEC(2, 1, 2, 4, 256, 8, 1)},
     /* M <= 4  */ {DEC(4, 1, 4, 4, 256, 6, 1), DEC(4, 1, 8, 4, 256, 4, 1), DEC(4, 1, 8, 2, 256, 6, 1), DEC(4, 1, 4, 8, 256, 4, 1)},
-    /* M <= 8  */ {DEC(8, 1, 4, 4, 256, 5, 1), DEC(8, 1, 8, 8, 256, 3, 4), DEC(8, 1, 8, 4, 256, 4, 4), DEC(8, 1, 4, 8, 256, 4, 1)},
-    /* M <= 16 */ {DEC(8, 2, 8, 4, 256, 3, 4), DEC(8, 2, 4, 4, 256, 4, 1), DEC(8, 2, 8, 2, 256, 4, 4), DEC(8, 2, 4, 2, 256, 4, 1)},
-    /* M > 16  */ {DEC(8, 4, 8, 2, 128, 5, 4), DEC(8, 4, 4, 2, 128, 6, 1), DEC(8, 4, 8, 1, 128, 6, 4), DEC(8, 4, 4, 1, 128, 6, 1)},
+    /* M <= 8  */ {DEC(8, 1, 4, 4, 256, 5, 1), DEC(8, 1, 8, 8, 256, 5, 4), DEC(8, 1, 8, 4, 256, 4, 4), DEC(8, 1, 4, 8, 256, 4, 1)},
+    /* M <= 16 */ {DEC(8, 2, 8, 4, 256, 3, 4), DEC(8, 2, 8, 4, 256, 6, 4), DEC(8, 2, 8, 2, 256, 4, 4), DEC(8, 2, 4, 4, 256, 4, 1)},
+    /* M > 16  */ {DEC(8, 4, 8, 2, 256, 5, 4), DEC(8, 4, 8, 2, 128, 5, 4), DEC(8, 4, 8, 1, 256, 4, 4), DEC(8, 4, 4, 2, 128, 6, 1)},
 };
 
 int m_class(int64_t M) { return M <= 1 ? 0 : M <= 2 ? 1 : M <= 4 ? 2 : M <= 8 ? 3 : M <= 16 ? 4 : 5; }
