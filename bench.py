@@ -1,0 +1,456 @@
+#!/usr/bin/env python
+"""Benchmark of the deterministic fused-upcast linear layer on B200.
+
+Workload (one "step"): the decode sweep on Llama-3-8B layer shapes -- M in {1,4,8,16,32} x
+(K,N) in {(4096,6144) qkv, (4096,4096) o, (4096,28672) gate_up, (14336,4096) down}: 20 calls of
+det_linear_run, each on its own seeded BF16 weight matrix (2.18 GB of weights per step, so every
+call finds its weights cold in L2).  Metric: BF16 weight bytes streamed per second (GB/s).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
+
+Prints ONE JSON line.  With --impl reference the CPU oracle is timed instead (host cores).
+Under torchrun every rank runs an independent replica on its own GPU (the path has no exchange
+step); the time is the maximum over ranks and `value` the aggregate over all ranks.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2609_25624_b200 import inputs  # noqa: E402
+
+METRIC = "decode weight streaming rate (BF16 weight bytes / s) over the Llama-3-8B decode sweep"
+UNIT = "GB/s"
+NOMINAL_SM_MHZ = 1965.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json, STREAM-style copy)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def fp32_peak_tflops(sm_count):
+    """CUDA-core FP32 peak: SMs x 128 lanes x 2 flop x max SM clock."""
+    return sm_count * 128 * 2 * NOMINAL_SM_MHZ * 1e6 / 1e12
+
+
+def decode_cases():
+    return [(M, N, K, name) for M in inputs.DECODE_MS for (name, K, N) in inputs.LLAMA3_8B_LAYER]
+
+
+def algorithmic_bytes(M, N, K):
+    """Bytes one call must move: W once (BF16), x once, y once, bias once."""
+    return 2 * N * K + 4 * M * K + 4 * M * N + 4 * N
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        if torch.cuda.is_available():
+            torch.cuda.set_device(local)
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return world, rank, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
+
+
+def max_over_ranks(value, world):
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([value], dtype=torch.float64, device="cuda" if torch.cuda.is_available() else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+    return value
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle
+# ---------------------------------------------------------------------------------------------
+def run_reference(args, world, rank):
+    if rank != 0:
+        return
+    from oracle import oracle
+    cases = decode_cases()
+    # bounded sample: every case of the sweep, restricted to the first `cols` weight rows, sized so
+    # that one step is a few seconds of host time
+    cols = args.ref_cols
+    data = []
+    for (M, N, K, name) in cases:
+        x, W, b = inputs.make_case(M, cols, K, seed=inputs.shape_seed(M, N, K))
+        data.append((x.numpy(), inputs.bf16_bits(W), b.numpy(), oracle.order_params(M, N, K)))
+    sample_bytes = sum(2 * cols * K for (_, _, K, _) in cases)
+    threads = oracle.threads()
+
+    def step():
+        for x, Wb, b, prm in data:
+            oracle.linear(x, Wb, b, params=prm)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = sample_bytes / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "Llama-3-8B decode sweep: M in {1,4,8,16,32} x {qkv,o,gate_up,down}, 20 calls/step",
+                   "sample": f"first {cols} weight rows of every case"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": f"all 20 cases of the sweep, first {cols} of N weight rows each, per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# own arm
+# ---------------------------------------------------------------------------------------------
+def time_graph(fn_capture, replays, stream):
+    """Capture fn_capture() into a CUDA graph on `stream`, replay it `replays` times and return the
+    best per-replay time in ms (CUDA events on the launching stream)."""
+    with torch.cuda.stream(stream):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            fn_capture()
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        best = float("inf")
+        for _ in range(replays):
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+    return best
+
+
+def run_own(args, world, rank, local):
+    from paper_2609_25624_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    props = torch.cuda.get_device_properties(dev)
+    hbm_peak, hbm_src = measured_peaks()
+    fp32_peak = fp32_peak_tflops(props.multi_processor_count)
+
+    cases = decode_cases()
+    st = torch.cuda.Stream()
+    work = []
+    for (M, N, K, name) in cases:
+        x, W, b = inputs.make_case(M, N, K)
+        plan = B.det_linear_plan(M, N, K)
+        work.append(dict(M=M, N=N, K=K, name=name, plan=plan, x=x.to(dev), W=W.to(dev), b=b.to(dev),
+                         y=torch.empty(M, N, dtype=torch.float32, device=dev),
+                         xh=x.pin_memory(), yh=torch.empty(M, N, dtype=torch.float32).pin_memory()))
+    weight_bytes = sum(2 * w["N"] * w["K"] for w in work)
+    alg_bytes = sum(algorithmic_bytes(w["M"], w["N"], w["K"]) for w in work)
+    flops = sum(2 * w["M"] * w["N"] * w["K"] for w in work)
+    launches_per_step = len(work)
+
+    def step():
+        for w in work:
+            B.det_linear_run(w["plan"], w["x"], w["W"], w["b"], w["y"])
+
+    with torch.cuda.stream(st):
+        for _ in range(2):          # eager warm-up (sets kernel attributes, builds tensor maps)
+            step()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=st):
+            step()
+        for _ in range(max(args.warmup, 3)):
+            graph.replay()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.5)             # let nvidia-smi come up so that its samples fall into the runs below
+        barrier(world)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_wall = time.perf_counter()
+        e0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        e1.record()
+        barrier(world)
+        ms_total = e0.elapsed_time(e1)
+        # the timed region may be shorter than the sampling period: keep the identical load running
+        # (untimed) until the sampler has seen about a second of it
+        extra = 0
+        while rank == 0 and time.perf_counter() - t_wall < 1.0:
+            for _ in range(50):
+                graph.replay()
+            torch.cuda.synchronize()
+            extra += 50
+        clocks = sampler.stop() if rank == 0 else None
+        if clocks is not None:
+            clocks["window"] = f"timed region plus {extra} untimed identical replays"
+        for w in work:
+            B.det_linear_plan_check(w["plan"])
+    ms_step = max_over_ranks(ms_total / args.steps, world)
+    value = world * weight_bytes / (ms_step * 1e-3) / 1e9
+
+    # ---- end to end: host activations in, host outputs back, every call ----
+    def step_host():
+        for w in work:
+            B.det_linear_run_host(w["plan"], w["xh"], w["W"], w["b"], w["yh"])
+
+    with torch.cuda.stream(st):
+        for _ in range(2):
+            step_host()
+        barrier(world)
+        t0 = time.perf_counter()
+        n_e2e = max(3, min(args.steps, 20))
+        for _ in range(n_e2e):
+            step_host()
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+    e2e_ms = max_over_ranks(e2e_ms, world)
+    e2e_value = world * weight_bytes / (e2e_ms * 1e-3) / 1e9
+    h2d = sum(4 * w["M"] * w["K"] for w in work)
+    d2h = sum(4 * w["M"] * w["N"] for w in work)
+
+    if rank != 0:
+        return
+
+    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "Llama-3-8B decode sweep: M in {1,4,8,16,32} x {qkv 4096->6144, o 4096->4096, "
+                               "gate_up 4096->28672, down 14336->4096}, 20 det_linear_run calls per step, bias present",
+                   "weights": "BF16 N(0,0.02^2) RNE, one seeded matrix per case (2.18 GB per step)",
+                   "activations": "FP32 N(0,1)", "l2": "inputs larger than L2: 2.18 GB of distinct weights between reuses",
+                   "launch": "one CUDA graph per step (programmatic dependent launch between the 20 kernels)",
+                   "multi_gpu": "replicas only (no exchange step in the path)"},
+        "pct_of_hbm_peak": 100.0 * value / world / hbm_peak,
+        "tflops_fp32": world * flops / (ms_step * 1e-3) / 1e12,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "note": "det_linear_run_host per call: x from pinned host memory, y back to host, weights resident"},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                     "traffic": None, "peak_source": hbm_src, "kernel": "decode_kernel (all 20 launches of a step)",
+                     "note": "M=16 and M=32 launches are FP32-FMA-bound on B200 (ridge 11.4 flop/B), see per_case"},
+    }
+
+    if not args.no_extras:
+        line["per_case"] = per_case_table(B, work, st, hbm_peak, fp32_peak)
+        line["prefill"] = prefill_table(B, dev, st, fp32_peak)
+        line["lm_head"] = lm_head_table(B, dev, st, hbm_peak, fp32_peak)
+        line["cpu_baseline"] = cpu_baseline(work)
+    else:
+        line["cpu_baseline"] = cpu_baseline(work)
+    traffic = os.path.join(ROOT, "profiles", "decode_dram_traffic.json")
+    if os.path.exists(traffic):
+        with open(traffic) as f:
+            line["roofline"]["traffic"] = json.load(f).get("bytes_per_step_launch_avg")
+    print(json.dumps(line), flush=True)
+    for w in work:
+        w["plan"].close()
+
+
+def per_case_table(B, work, st, hbm_peak, fp32_peak):
+    """Per-call times with cold weights: each case replays a graph that cycles through clones of its
+    weight matrix totalling >= 512 MB."""
+    rows = []
+    for w in work:
+        M, N, K = w["M"], w["N"], w["K"]
+        wbytes = 2 * N * K
+        R = max(2, -(-(512 << 20) // wbytes))
+        Ws = [w["W"]] + [w["W"].clone() for _ in range(R - 1)]
+        plans = [B.det_linear_plan(M, N, K) for _ in range(R)]
+        reps = R * max(1, 16 // R)
+        with torch.cuda.stream(st):
+            for i in range(R):
+                B.det_linear_run(plans[i], w["x"], Ws[i], w["b"], w["y"])
+            torch.cuda.synchronize()
+        ms = time_graph(lambda: [B.det_linear_run(plans[i % R], w["x"], Ws[i % R], w["b"], w["y"]) for i in range(reps)],
+                        5, st) / reps
+        for p in plans:
+            p.close()
+        del Ws
+        t_hbm = wbytes / (hbm_peak * 1e9)
+        t_fma = 2 * M * N * K / (fp32_peak * 1e12)
+        rows.append({"name": w["name"], "M": M, "N": N, "K": K, "us": ms * 1e3, "weight_gbs": wbytes / ms / 1e6,
+                     "pct_hbm": 100 * wbytes / ms / 1e6 / hbm_peak, "tflops": 2 * M * N * K / ms / 1e9,
+                     "pct_fp32": 100 * 2 * M * N * K / ms / 1e9 / fp32_peak,
+                     "bound": "hbm" if t_hbm >= t_fma else "fp32", "pct_of_roofline": 100 * max(t_hbm, t_fma) / (ms * 1e-3)})
+    return rows
+
+
+def prefill_table(B, dev, st, fp32_peak):
+    rows = []
+    for (name, K, N) in inputs.PREFILL_SHAPES:
+        W = None
+        for M in inputs.PREFILL_MS:
+            x, Wc, b = inputs.make_case(M, N, K)
+            if W is None:
+                W = Wc.to(dev)          # timing does not depend on the weight values: one matrix per shape
+            xd, bd = x.to(dev), b.to(dev)
+            y = torch.empty(M, N, dtype=torch.float32, device=dev)
+            plan = B.det_linear_plan(M, N, K)
+            with torch.cuda.stream(st):
+                B.det_linear_run(plan, xd, W, bd, y)
+                torch.cuda.synchronize()
+            ms = time_graph(lambda: B.det_linear_run(plan, xd, W, bd, y), 3, st)
+            B.det_linear_plan_check(plan)
+            prm = B.det_linear_plan_get_params(plan)
+            plan.close()
+            tf = 2 * M * N * K / ms / 1e9
+            rows.append({"name": name, "M": M, "N": N, "K": K, "S": prm.S, "us": ms * 1e3, "tflops": tf,
+                         "pct_fp32_peak": 100 * tf / fp32_peak})
+    total_flops = sum(2 * r["M"] * r["N"] * r["K"] for r in rows)
+    total_s = sum(r["us"] for r in rows) * 1e-6
+    return {"fp32_peak_tflops": fp32_peak, "peak_source": "148 SMs x 128 lanes x 2 x 1965 MHz (derived)",
+            "aggregate_tflops": total_flops / total_s / 1e12, "aggregate_pct_fp32_peak": 100 * total_flops / total_s / 1e12 / fp32_peak,
+            "cases": rows}
+
+
+def lm_head_table(B, dev, st, hbm_peak, fp32_peak):
+    name, K, N = inputs.LLAMA3_8B_LM_HEAD
+    rows = []
+    W = inputs.make_weight(N, K, inputs.named_seed("lm_head")).to(dev)
+    W2 = W.clone()
+    for M in inputs.LM_HEAD_MS:
+        g = torch.Generator().manual_seed(inputs.shape_seed(M, N, K))
+        x = torch.randn(M, K, generator=g).to(dev)
+        y = torch.empty(M, N, dtype=torch.float32, device=dev)
+        idx = torch.empty(M, dtype=torch.int32, device=dev)
+        plans = [B.det_linear_plan(M, N, K) for _ in range(2)]
+
+        def call():
+            B.det_linear_run(plans[0], x, W, None, y)
+            B.det_argmax_rows(y, idx)
+            B.det_linear_run(plans[1], x, W2, None, y)
+            B.det_argmax_rows(y, idx)
+        with torch.cuda.stream(st):
+            call()
+            torch.cuda.synchronize()
+        ms = time_graph(call, 3, st) / 2
+        for p in plans:
+            p.close()
+        wbytes = 2 * N * K
+        rows.append({"M": M, "us_linear_plus_argmax": ms * 1e3, "weight_gbs": wbytes / ms / 1e6,
+                     "pct_hbm": 100 * wbytes / ms / 1e6 / hbm_peak, "tflops": 2 * M * N * K / ms / 1e9,
+                     "pct_fp32": 100 * 2 * M * N * K / ms / 1e9 / fp32_peak})
+    return rows
+
+
+def cpu_baseline(work):
+    """The oracle as it stands, on the host cores, on a bounded sample of the same step."""
+    from oracle import oracle
+    cols = 512
+    data = []
+    for w in work:
+        xs = w["xh"].numpy()
+        Wb = inputs.bf16_bits(w["W"][:cols].cpu())
+        data.append((xs, Wb, w["b"][:cols].cpu().numpy(), oracle.order_params(w["M"], w["N"], w["K"])))
+    oracle.linear(*data[0][:3], params=data[0][3])          # load the library
+    t0 = time.perf_counter()
+    for x, Wb, b, prm in data:
+        oracle.linear(x, Wb, b, params=prm)
+    dt = time.perf_counter() - t0
+    sample_bytes = sum(2 * cols * w["K"] for w in work)
+    return {"value": sample_bytes / dt / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"all 20 cases of the step, first {cols} of N weight rows each (one pass, {dt:.2f} s)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the per-case, prefill and LM-head tables")
+    ap.add_argument("--ref-cols", type=int, default=512, help="weight rows per case in the reference arm's sample")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        world = int(os.environ.get("WORLD_SIZE", "1"))
+        rank = int(os.environ.get("RANK", "0"))
+        run_reference(args, world, rank)
+        return
+    world, rank, local = dist_setup(args.gpus)
+    try:
+        run_own(args, world, rank, local)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

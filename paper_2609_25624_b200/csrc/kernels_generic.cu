@@ -3,6 +3,7 @@
 // the paper's ragged probe), the split-K second pass and the row argmax.  They are not tuned.
 #include "internal.h"
 #include "device_utils.cuh"
+#include <cooperative_groups.h>
 
 namespace detlin {
 
@@ -114,9 +115,14 @@ cudaError_t launch_combine(const LaunchArgs& a)
     return cudaGetLastError();
 }
 
-// Row argmax, lowest index on ties (the paper's stated tie rule for greedy decoding).  One block
-// per row.  Ordering key: NaN beats everything (first NaN wins), otherwise larger value, then
-// smaller index.  Comparisons only, so the result is exact and order-free.
+// Row argmax, lowest index on ties (the paper's stated tie rule for greedy decoding).  Ordering
+// key: NaN beats everything (first NaN wins), otherwise larger value, then smaller index.
+// Comparisons only, so the result is exact and order-free.  A cluster of kArgmaxCluster blocks
+// shares one row: each block scans a contiguous slice, the partial results meet in block 0 of the
+// cluster through distributed shared memory (hardware cluster barrier, no spinning).
+namespace cg = cooperative_groups;
+constexpr int kArgmaxCluster = 8;
+
 __device__ __forceinline__ bool argmax_better(float v, int i, float bv, int bi)
 {
     const bool vn = (v != v), bn = (bv != bv);
@@ -124,38 +130,58 @@ __device__ __forceinline__ bool argmax_better(float v, int i, float bv, int bi)
     return (v > bv) || (v == bv && i < bi);
 }
 
-__global__ void __launch_bounds__(1024)
-argmax_rows_kernel(const float* __restrict__ y, int64_t N, int32_t* __restrict__ idx)
+__device__ __forceinline__ void argmax_warp(float& bv, int& bi)
 {
-    __shared__ float sv[32];
-    __shared__ int si[32];
-    const float* row = y + (int64_t)blockIdx.x * N;
-    float bv = row[0];
-    int bi = 0;
-    for (int64_t n = threadIdx.x; n < N; n += blockDim.x) {
-        const float v = row[n];
-        if (argmax_better(v, (int)n, bv, bi)) { bv = v; bi = (int)n; }
-    }
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
         const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
         if (argmax_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
     }
+}
+
+__global__ void __cluster_dims__(kArgmaxCluster, 1, 1) __launch_bounds__(1024)
+argmax_rows_kernel(const float* __restrict__ y, int64_t N, int32_t* __restrict__ idx)
+{
+    __shared__ float sv[32];
+    __shared__ int si[32];
+    __shared__ float block_v;
+    __shared__ int block_i;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const float* row = y + (int64_t)blockIdx.y * N;
+    const int64_t per = (N + kArgmaxCluster - 1) / kArgmaxCluster;
+    const int64_t lo = rank * per;
+    const int64_t hi = (lo + per < N) ? lo + per : N;
+    // a block whose slice is empty contributes the row's first element (always a valid candidate)
+    float bv = row[lo < N ? lo : 0];
+    int bi = (int)(lo < N ? lo : 0);
+    for (int64_t n = lo + threadIdx.x; n < hi; n += blockDim.x) {
+        const float v = row[n];
+        if (argmax_better(v, (int)n, bv, bi)) { bv = v; bi = (int)n; }
+    }
+    argmax_warp(bv, bi);
     if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
     __syncthreads();
     if (threadIdx.x < 32) {
         const int nw = blockDim.x >> 5;
         bv = (threadIdx.x < nw) ? sv[threadIdx.x] : sv[0];
         bi = (threadIdx.x < nw) ? si[threadIdx.x] : si[0];
-#pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
+        argmax_warp(bv, bi);
+        if (threadIdx.x == 0) { block_v = bv; block_i = bi; }
+    }
+    cluster.sync();
+    if (rank == 0 && threadIdx.x == 0) {
+        bv = block_v;
+        bi = block_i;
+        for (int r = 1; r < kArgmaxCluster; ++r) {
+            const float ov = *cluster.map_shared_rank(&block_v, r);
+            const int oi = *cluster.map_shared_rank(&block_i, r);
             if (argmax_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
         }
-        if (threadIdx.x == 0) idx[blockIdx.x] = bi;
+        idx[blockIdx.y] = bi;
     }
+    cluster.sync();     // keep every block's shared memory alive until block 0 has read it
 }
 
 cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cudaStream_t stream)
@@ -163,7 +189,8 @@ cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cu
     const int64_t max_rows = 65535;
     for (int64_t m0 = 0; m0 < M; m0 += max_rows) {
         const int64_t mm = (M - m0 < max_rows) ? M - m0 : max_rows;
-        argmax_rows_kernel<<<(unsigned)mm, 1024, 0, stream>>>(y + m0 * N, N, idx + m0);
+        dim3 grid(kArgmaxCluster, (unsigned)mm);
+        argmax_rows_kernel<<<grid, 1024, 0, stream>>>(y + m0 * N, N, idx + m0);
     }
     return cudaGetLastError();
 }
