@@ -307,6 +307,7 @@ def run_own(args, world, rank, local):
                      "note": "M=16 and M=32 launches are FP32-FMA-bound on B200 (ridge 11.4 flop/B), see per_case"},
     }
 
+    line["calibration"] = calibration(B, dev, fp32_peak)
     if not args.no_extras:
         line["per_case"] = per_case_table(B, work, st, hbm_peak, fp32_peak)
         line["prefill"] = prefill_table(B, dev, st, fp32_peak)
@@ -321,6 +322,19 @@ def run_own(args, world, rank, local):
     print(json.dumps(line), flush=True)
     for w in work:
         w["plan"].close()
+
+
+def calibration(B, dev, fp32_peak):
+    """Denominators measured on this device in this run: FP32 FMA issue peak of the CUDA cores and
+    read-only HBM streaming bandwidth (the driver-written copy bandwidth is a read+write figure)."""
+    buf = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+    buf.fill_(1)
+    out = {"fp32_peak_derived_tflops": fp32_peak,
+           "fp32_fma_measured_tflops": B.det_test_measure_fma_peak(False),
+           "fp32_fma2_measured_tflops": B.det_test_measure_fma_peak(True),
+           "hbm_read_only_measured_gbs": B.det_test_measure_read_bandwidth(buf)}
+    del buf
+    return out
 
 
 def per_case_table(B, work, st, hbm_peak, fp32_peak):

@@ -38,6 +38,17 @@ DET_API det_status_t det_test_green_stream_create(int sm_count, void** stream_ou
                                           int* sm_granted);
 DET_API void det_test_green_stream_destroy(void* handle);
 
+/*
+ * Calibration for the benchmark's rooflines (these compute nothing of the method).
+ * det_test_measure_fma_peak: FP32 multiply-add issue peak of the CUDA cores in TFLOP/s, measured
+ * with a register-only loop of scalar fma.rn.f32 (packed = 0) or fma.rn.f32x2 (packed = 1).
+ * det_test_measure_read_bandwidth: read-only streaming rate in GB/s over `bytes` of device memory
+ * at `buf` (16-byte aligned, at least 1 MiB; use a buffer much larger than L2).
+ * Both run on the default stream and synchronise.
+ */
+DET_API det_status_t det_test_measure_fma_peak(int packed, double* tflops_out);
+DET_API det_status_t det_test_measure_read_bandwidth(const void* buf, size_t bytes, double* gbs_out);
+
 #ifdef __cplusplus
 }
 #endif

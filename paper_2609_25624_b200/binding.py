@@ -78,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.det_test_green_stream_create.restype = i32
         L.det_test_green_stream_destroy.argtypes = [p]
         L.det_test_green_stream_destroy.restype = None
+        L.det_test_measure_fma_peak.argtypes = [i32, ctypes.POINTER(ctypes.c_double)]
+        L.det_test_measure_fma_peak.restype = i32
+        L.det_test_measure_read_bandwidth.argtypes = [p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_double)]
+        L.det_test_measure_read_bandwidth.restype = i32
         _lib = L
     return _lib
 
@@ -217,3 +221,17 @@ def det_test_green_stream_create(sm_count: int):
 
 def det_test_green_stream_destroy(handle) -> None:
     lib().det_test_green_stream_destroy(handle)
+
+
+def det_test_measure_fma_peak(packed: bool) -> float:
+    """Measured FP32 FMA issue peak of the CUDA cores in TFLOP/s (scalar or packed FP32x2)."""
+    out = ctypes.c_double(0.0)
+    _check(lib().det_test_measure_fma_peak(1 if packed else 0, ctypes.byref(out)))
+    return out.value
+
+
+def det_test_measure_read_bandwidth(buf) -> float:
+    """Read-only streaming bandwidth in GB/s over a CUDA tensor (use one much larger than L2)."""
+    out = ctypes.c_double(0.0)
+    _check(lib().det_test_measure_read_bandwidth(buf.data_ptr(), buf.numel() * buf.element_size(), ctypes.byref(out)))
+    return out.value
