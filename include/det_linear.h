@@ -137,6 +137,30 @@ DET_API void det_linear_plan_destroy(det_linear_plan_t* plan);
  */
 DET_API det_status_t det_argmax_rows(const float* y, int64_t M, int64_t N, int32_t* idx, void* stream);
 
+/*
+ * The same computation for callers that cannot allocate (the paper has no counterpart for this
+ * entry point).  A host that owns all device memory through its own pool or arena, a plugin that
+ * may not allocate after initialisation, or a latency-critical loop that cannot afford the
+ * implicit synchronisation of an allocation can use this call instead of det_linear_plan +
+ * det_linear_run: it calls no cudaMalloc / cudaFree and no allocating library routine, and keeps no
+ * plan.  Inputs and output are passed as for det_linear_run (device pointers, same layouts, b may
+ * be NULL); the result has the same bits.
+ *
+ * The split-K partials (needed only when the shape splits K, i.e. S > 1: 4*S*M*N bytes) live in a
+ * 4 MiB array built into the library image, present on every GPU that loads the library until the
+ * process exits.  A shape that needs more is rejected with DET_ERR_UNSUPPORTED_SHAPE and a message
+ * that names both sizes; nothing is launched then.  All calls share that one array and it keeps the
+ * last call's contents (nothing in it needs clearing: each call overwrites what it reads), so two
+ * calls whose GPU work overlaps -- different streams, or different host threads -- race on it:
+ * issue them on one stream or order them yourself.
+ *
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call before starting any stream capture.  The kernels are the library's generic
+ * ones (any shape and alignment, not tuned for speed).  Enqueues on `stream`, no synchronisation.
+ */
+DET_API det_status_t det_linear_run_noalloc(int64_t M, int64_t N, int64_t K, const float* x, const uint16_t* W,
+                                            const float* b, float* y, void* stream);
+
 /* Message of the last error on the calling thread ("" if none).  Never NULL. */
 DET_API const char* det_last_error(void);
 

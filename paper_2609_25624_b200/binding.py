@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.det_test_green_stream_create.restype = i32
         L.det_test_green_stream_destroy.argtypes = [p]
         L.det_test_green_stream_destroy.restype = None
+        L.det_linear_run_noalloc.argtypes = [i64, i64, i64, p, p, p, p, p]
+        L.det_linear_run_noalloc.restype = i32
         L.det_test_measure_fma_peak.argtypes = [i32, ctypes.POINTER(ctypes.c_double)]
         L.det_test_measure_fma_peak.restype = i32
         L.det_test_measure_read_bandwidth.argtypes = [p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_double)]
@@ -186,6 +188,22 @@ def det_linear_run_host(plan: Plan, x_host, W, b, y_host, stream=None) -> None:
     _check(lib().det_linear_run_host(plan.handle, x_host.data_ptr(), W.data_ptr(),
                                      b.data_ptr() if b is not None else None, y_host.data_ptr(),
                                      _stream_ptr(stream)))
+
+
+def det_linear_run_noalloc(x, W, b, y, stream=None) -> None:
+    """The same linear layer without any allocation (no plan; split-K partials in the library's
+    built-in 4 MiB scratch).  For callers that must not allocate: hosts that own all device memory
+    through their own pool, plugins after initialisation, latency-critical loops.  Calls whose GPU
+    work overlaps race on the shared scratch."""
+    M, K = x.shape
+    N = W.shape[0]
+    _expect(x, torch.float32, (M, K), "x")
+    _expect(W, torch.bfloat16, (N, K), "W")
+    _expect(y, torch.float32, (M, N), "y")
+    if b is not None:
+        _expect(b, torch.float32, (N,), "b")
+    _check(lib().det_linear_run_noalloc(M, N, K, x.data_ptr(), W.data_ptr(), b.data_ptr() if b is not None else None,
+                                        y.data_ptr(), _stream_ptr(stream)))
 
 
 def det_linear_plan_check(plan: Plan, stream=None) -> None:
