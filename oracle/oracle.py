@@ -53,7 +53,7 @@ def order_params(M: int, N: int, K: int) -> dict:
     if min(M, N, K) < 1:
         raise ValueError("M, N, K must be >= 1")
     if M <= DECODE_MAX_M:
-        bucket, V, L, P = "decode", 4, 32, 2
+        bucket, V, L, P = "decode", 4, 32, 1
     else:
         bucket, V, L, P = "prefill", 2, 1, 2
     s_req = split_request(M, N, K)

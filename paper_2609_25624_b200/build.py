@@ -14,7 +14,8 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libdet_linear.so")
 OBJ_DIR = os.path.join(HERE, "csrc", "obj")
 
-SOURCES = ["plan.cpp", "capi.cu", "kernels_generic.cu", "kernels_decode.cu", "kernels_prefill.cu", "bench_kernels.cu", "noalloc.cu"]
+SOURCES = ["plan.cpp", "capi.cu", "kernels_generic.cu", "kernels_decode.cu", "decode_inst_0.cu", "decode_inst_1.cu", "decode_inst_2.cu",
+           "decode_inst_3.cu", "kernels_prefill.cu", "bench_kernels.cu", "noalloc.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

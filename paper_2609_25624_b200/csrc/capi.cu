@@ -270,9 +270,12 @@ det_status_t det_test_plan_set_max_blocks(det_linear_plan_t* plan, int max_block
 det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
 {
     if (!plan || variant < 0) { set_error("set_variant: bad argument"); return DET_ERR_INVALID_ARG; }
-    if (plan->prm.bucket == 0 && variant > decode_num_variants()) {
-        set_error("set_variant: decode kernel has %d variants", decode_num_variants());
-        return DET_ERR_INVALID_ARG;
+    if (plan->prm.bucket == 0) {
+        DecodeConfig cfg;
+        if (!decode_config_for(plan->prm.M, plan->prm.N, plan->prm.K, variant, &cfg)) {
+            set_error("set_variant: the decode kernel has fewer than %d tilings for this batch size", variant);
+            return DET_ERR_INVALID_ARG;
+        }
     }
     plan->variant = variant;
     return DET_OK;

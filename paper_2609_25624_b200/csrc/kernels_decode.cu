@@ -1,460 +1,77 @@
-// Decode kernel (bucket M <= 64): streams BF16 weight tiles from HBM through a TMA -> shared-memory
-// ring, widens them to FP32 in registers (Eq. 2) and accumulates with packed IEEE FP32 FMAs
-// (fma.rn.f32x2; rule R1) in the frozen decode order (V=4, L=32, P=2):
-//
-//   lane l of a warp owns k = c + 4l + j (j = 0..3) of every 128-element chunk c; its even
-//   elements feed sub-chain 0 and its odd elements sub-chain 1, which are exactly the two halves
-//   of one FP32x2 accumulator; the 64 leaves of an output are then summed adjacent-first
-//   (sub-chains inside the lane, then lanes xor 1, 2, 4, 8, 16).
-//
-// Everything else is schedule and therefore numerically inert (supplement C on rule R2: tile
-// sizes, warp counts and pipeline depth do not change the reduction tree): one producer warp
-// issues the bulk-tensor copies, WM x WR consumer warps each own an (MT batch rows) x (RT weight
-// rows) register tile, thread blocks walk (row tile, segment, batch block) work units in a strided
-// loop.  Rule R4 holds by construction: nothing that touches the order reads M.
-//
-// Every wait on a completion barrier is bounded; a wait that expires records the fact in the
-// plan's device status word and the block drains and returns.
-#include "internal.h"
-#include "device_utils.cuh"
+// Decode kernel dispatch: picks one of the compiled tilings for a shape.  The choice only changes
+// the schedule (tile sizes, warp counts and ring depth are numerically inert: supplement C on
+// rule R2), so it may read the SM count and the occupancy; the reduction order never does.
+#include "decode_kernel.cuh"
 
 namespace detlin {
 
 namespace {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
-constexpr unsigned kTryWaitHintNs = 2000;                   // a waiting thread may sleep this long per try
+using decode_detail::DecodeEntry;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+const DecodeClassTable* class_table(int cls)
 {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+    static const DecodeClassTable* const t[6] = {&kDecodeClass0, &kDecodeClass1, &kDecodeClass2,
+                                                 &kDecodeClass3, &kDecodeClass4, &kDecodeClass5};
+    return t[cls];
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(kTryWaitHintNs)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ float4 lds128(uint32_t addr)
-{
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ uint2 lds64(uint32_t addr)
-{
-    uint2 v;
-    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ unsigned long long global_timer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait.  Returns false if the block is aborting or the wait expired (then it marks the
-// block as aborting and records the site in the device status word).
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
-                                           unsigned site)
-{
-    const unsigned long long t0 = global_timer_ns();
-    for (;;) {
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
-            *abort_flag = 1;
-            atomicExch(&status->where, site);
-            atomicExch(&status->timeout_flag, 1u);
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
-                                          unsigned site)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status, site);
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
-                                            unsigned long long policy)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
-        " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
-        "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
-        : "memory");
-}
-
-// PG = warps in the producer group: 1 (plain) or 4 (a whole warpgroup, which lets the kernel move
-// registers from the producer to the consumers with setmaxnreg when the consumer tile is large).
-template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
-struct Cfg {
-    static constexpr int kConsumerWarps = WM * WR;
-    static constexpr int kThreads = (kConsumerWarps + PG) * 32;
-    static constexpr int kMB = MT * WM;                       // batch rows per x box
-    static constexpr int kRB = RT * WR;                       // weight rows per block tile
-    static constexpr int kXBytes = kMB * KC * 4;
-    static constexpr int kWBoxBytes = RT * KC * 2;
-    static constexpr int kStageBytes = kXBytes + WR * kWBoxBytes;
-    static constexpr int kBarBytes = 256;                     // 2*STAGES barriers + abort flag
-    static constexpr int kSmemBytes = STAGES * kStageBytes + kBarBytes + 128;   // +128 for alignment
-    // With a producer warpgroup the block is compiled for kMinBlocks blocks per SM and then moves
-    // registers inside its own allocation (threads x launch registers): producers shrink to
-    // kProducerRegs, consumers grow to kConsumerRegs.  setmaxnreg.inc blocks until the registers
-    // exist, so the request must never exceed what the block owns.
-    static constexpr int kMinBlocks = (PG == 4 && kConsumerWarps == 4) ? 2 : 1;
-    static constexpr int kLaunchRegsRaw = (65536 / (kMinBlocks * kThreads)) / 8 * 8;
-    static constexpr int kLaunchRegs = kLaunchRegsRaw > 255 ? 248 : kLaunchRegsRaw;
-    static constexpr int kProducerRegs = 32;
-    static constexpr int kConsumerRegsRaw =
-        PG == 4 ? ((kThreads * kLaunchRegs - PG * 32 * kProducerRegs) / (kConsumerWarps * 32)) / 8 * 8 : 0;
-    static constexpr int kConsumerRegs = kConsumerRegsRaw > 240 ? 240 : kConsumerRegsRaw;
-    static_assert(PG == 1 || kConsumerRegs * kConsumerWarps * 32 + kProducerRegs * PG * 32 <= kThreads * kLaunchRegs,
-                  "register move must fit in the block's own allocation");
-    static_assert(PG == 1 || kConsumerRegs >= kLaunchRegs, "consumers only ever grow");
-    static_assert(PG == 1 || (PG == 4 && kConsumerWarps % 4 == 0), "setmaxnreg works on whole warpgroups");
-    static_assert(STAGES >= 2 && STAGES <= 12, "ring depth");
-    static_assert(KC % 128 == 0 && KC <= 256, "a stage holds whole 128-element chunks; TMA boxes are <= 256 wide");
-    static_assert(kXBytes % 128 == 0 && kWBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
-};
-
-// Butterfly reduce-scatter over the 32 lanes that realises the adjacent-first tree: at step i
-// lanes l and l ^ (1 << i) exchange halves of their value arrays and add, so each lane ends with
-// NV/32 (at least 1) tree roots.  Lane with bit i set keeps the upper half at step i.
-template <int NV>
-__device__ __forceinline__ void lane_tree_scatter(float (&v)[NV], int lane)
-{
-    int n = NV;
-#pragma unroll
-    for (int i = 0; i < 5; ++i) {
-        const int d = 1 << i;
-        if (n > 1) {
-            const int half = n >> 1;
-            const bool hi = (lane >> i) & 1;
-#pragma unroll
-            for (int t = 0; t < NV / 2; ++t) {
-                if (t < half) {
-                    const float send = hi ? v[t] : v[t + half];
-                    const float keep = hi ? v[t + half] : v[t];
-                    v[t] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, d));
-                }
-            }
-            n = half;
-        } else {
-            v[0] = __fadd_rn(v[0], __shfl_xor_sync(0xffffffffu, v[0], d));
-        }
-    }
-}
-
-template <int REGS>
-__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS)); }
-template <int REGS>
-__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS)); }
-
-// Programmatic dependent launch: let the next kernel in the stream start its prologue early, and
-// wait for the previous kernel's results before touching anything it may have produced.
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-struct Unit {
-    int tile, s, mb, k_lo, k_hi;
-};
-__device__ __forceinline__ Unit decode_unit(long long u, int n_row_tiles, int S, int seg_len, int K)
-{
-    Unit r;
-    r.tile = (int)(u % n_row_tiles);
-    const long long q = u / n_row_tiles;
-    r.s = (int)(q % S);
-    r.mb = (int)(q / S);
-    r.k_lo = r.s * seg_len;
-    r.k_hi = min(K, r.k_lo + seg_len);
-    return r;
-}
-
-template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
-__global__ void __launch_bounds__((WM * WR + PG) * 32, (Cfg<MT, WM, RT, WR, KC, STAGES, PG>::kMinBlocks))
-decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-              const float* __restrict__ bias, float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct,
-              int n_row_tiles, int n_mblocks, DeviceStatus* status)
-{
-    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG>;
-    extern __shared__ unsigned char smem_raw[];
-    // 128-byte aligned base (TMA destination requirement)
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
-    const uint32_t smem_base = smem_u32(smem);
-    unsigned char* bar_mem = smem + STAGES * C::kStageBytes;
-    const uint32_t full0 = smem_u32(bar_mem);                 // full[s]  at full0 + 8 s
-    const uint32_t empty0 = full0 + 8 * STAGES;               // empty[s] at empty0 + 8 s
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 16 * STAGES);
-
-    const int warp = threadIdx.x >> 5;
-    const int lane = threadIdx.x & 31;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, C::kConsumerWarps);
-        }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
-    pdl_launch_dependents();
-
-    const long long total_units = (long long)n_row_tiles * S * n_mblocks;
-
-    if (warp < PG) {
-        // ---------------- producer group: one lane issues all bulk-tensor copies ----------------
-        if (PG == 4) reg_dec<C::kProducerRegs>();
-        if (warp == 0 && lane == 0) {
-            unsigned long long pol_w, pol_x;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_w));
-            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_x));
-            unsigned it = 0;
-            bool ok = true;
-            // Weights never depend on the previous kernel, activations may: the first ring of
-            // weight boxes is requested before waiting for the previous kernel to finish.
-            unsigned pre = 0;
-            {
-                long long u = blockIdx.x;
-                unsigned j = 0;
-                while (u < total_units && j < (unsigned)STAGES) {
-                    const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
-                    for (int k0 = un.k_lo; k0 < un.k_hi && j < (unsigned)STAGES; k0 += KC, ++j) {
-                        const uint32_t fb = full0 + 8 * j;
-                        mbar_arrive_expect_tx(fb, C::kStageBytes);
-                        const uint32_t sbase = smem_u32(smem + j * C::kStageBytes);
-#pragma unroll
-                        for (int wr = 0; wr < WR; ++wr)
-                            tma_load_2d(sbase + C::kXBytes + wr * C::kWBoxBytes, &map_w, k0, un.tile * C::kRB + wr * RT, fb, pol_w);
-                    }
-                    u += gridDim.x;
-                }
-                pre = j;
-            }
-            pdl_wait();
-            for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
-                const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
-                const int n0 = un.tile * C::kRB;
-                for (int k0 = un.k_lo; k0 < un.k_hi; k0 += KC, ++it) {
-                    const int st = it % STAGES;
-                    const unsigned use = it / STAGES;
-                    const uint32_t fb = full0 + 8 * st;
-                    const uint32_t sbase = smem_u32(smem + st * C::kStageBytes);
-                    if (it >= pre) {
-                        if (use > 0 && !mbar_wait(empty0 + 8 * st, (use - 1) & 1, abort_flag, status, 1)) { ok = false; break; }
-                        mbar_arrive_expect_tx(fb, C::kStageBytes);
-#pragma unroll
-                        for (int wr = 0; wr < WR; ++wr)
-                            tma_load_2d(sbase + C::kXBytes + wr * C::kWBoxBytes, &map_w, k0, n0 + wr * RT, fb, pol_w);
-                    }
-                    tma_load_2d(sbase, &map_x, k0, un.mb * C::kMB, fb, pol_x);
-                }
-            }
-            if (!ok) {
-                // aborting: wait (bounded) for the copies this thread still has in flight
-                const unsigned first = it > (unsigned)STAGES ? it - STAGES : 0u;
-                for (unsigned j = first; j < it; ++j) {
-                    const unsigned long long t0 = global_timer_ns();
-                    while (!mbar_try_wait(full0 + 8 * (j % STAGES), (j / STAGES) & 1))
-                        if (global_timer_ns() - t0 > kWaitLimitNs) break;
-                }
-            }
-        }
-    } else {
-        // ---------------- consumer warps ----------------
-        if (PG == 4) reg_inc<C::kConsumerRegs>();
-        const int cw = warp - PG;
-        const int wm = cw % WM;
-        const int wr = cw / WM;
-        unsigned it = 0;
-        bool ok = true;
-        bool waited = false;
-        for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
-            const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
-
-            float2 acc[MT][RT];          // (even-k sub-chain, odd-k sub-chain) of the lane's leaf pair
-#pragma unroll
-            for (int m = 0; m < MT; ++m)
-#pragma unroll
-                for (int q = 0; q < RT; ++q) acc[m][q] = make_float2(0.0f, 0.0f);
-
-            for (int k0 = un.k_lo; k0 < un.k_hi; k0 += KC, ++it) {
-                const int st = it % STAGES;
-                if (!mbar_wait(full0 + 8 * st, (it / STAGES) & 1, abort_flag, status, 2)) { ok = false; break; }
-                const uint32_t xs = smem_base + st * C::kStageBytes + (wm * MT) * (KC * 4) + lane * 16;
-                const uint32_t ws = smem_base + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * 8;
-#pragma unroll(MT * RT >= 64 ? 1 : 2)
-                for (int cc = 0; cc < KC / 128; ++cc) {
-                    // Elements beyond the end of K are skipped, not zero-filled (K % 4 == 0 here, so a
-                    // lane's four elements are all inside or all outside).  Whole chunks take the
-                    // warp-uniform branch.
-                    const int kc0 = k0 + cc * 128;
-                    if (kc0 + 128 <= un.k_hi || kc0 + 4 * lane < un.k_hi) {
-                        float2 wp[RT][2];
-#pragma unroll
-                        for (int q = 0; q < RT; ++q) {
-                            const uint2 w = lds64(ws + q * (KC * 2) + cc * 256);
-                            wp[q][0] = make_float2(up_lo(w.x), up_hi(w.x));
-                            wp[q][1] = make_float2(up_lo(w.y), up_hi(w.y));
-                        }
-#pragma unroll
-                        for (int m = 0; m < MT; ++m) {
-                            const float4 xv = lds128(xs + m * (KC * 4) + cc * 512);
-                            const float2 x01 = make_float2(xv.x, xv.y), x23 = make_float2(xv.z, xv.w);
-#pragma unroll
-                            for (int q = 0; q < RT; ++q) acc[m][q] = __ffma2_rn(x01, wp[q][0], acc[m][q]);
-#pragma unroll
-                            for (int q = 0; q < RT; ++q) acc[m][q] = __ffma2_rn(x23, wp[q][1], acc[m][q]);
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * st);
-            }
-            if (!ok) break;
-
-            // ---- epilogue: sub-chains, lane tree, bias, store ----
-            float v[MT * RT];
-#pragma unroll
-            for (int m = 0; m < MT; ++m)
-#pragma unroll
-                for (int q = 0; q < RT; ++q) v[m * RT + q] = __fadd_rn(acc[m][q].x, acc[m][q].y);
-            lane_tree_scatter<MT * RT>(v, lane);
-            constexpr int NV = MT * RT;
-            constexpr int kKeep = NV >= 32 ? NV / 32 : 1;
-            // index of v[0] in the (m, q) tile: bit i of the lane selected the upper half at step i
-            int base = 0;
-            {
-                int n = NV;
-#pragma unroll
-                for (int i = 0; i < 5; ++i)
-                    if (n > 1) { n >>= 1; base += ((lane >> i) & 1) * n; }
-            }
-            // with fewer than 32 values the lanes that differ only in their high bits hold the same root;
-            // the one whose high bits are zero stores it
-            constexpr int kLog2NV = NV >= 32 ? 5 : NV == 16 ? 4 : NV == 8 ? 3 : NV == 4 ? 2 : NV == 2 ? 1 : 0;
-            const bool owner = (lane >> kLog2NV) == 0;
-            // the output buffer may still be read by the previous kernel in the stream
-            if (!waited) { pdl_wait(); waited = true; }
-            if (owner) {
-#pragma unroll
-                for (int t = 0; t < kKeep; ++t) {
-                    const int idx = base + t;
-                    const int m = un.mb * C::kMB + wm * MT + idx / RT;
-                    const int n = un.tile * C::kRB + wr * RT + idx % RT;
-                    if (m < M && n < N) {
-                        float r0 = v[t];
-                        if (direct) {
-                            if (bias) r0 = __fadd_rn(r0, bias[n]);
-                            out[(long long)m * N + n] = r0;
-                        } else {
-                            out[((long long)un.s * M + m) * N + n] = r0;
-                        }
-                    }
-                }
-            }
-        }
-    }
-    __syncthreads();
-}
-
-typedef cudaError_t (*DecodeLaunchFn)(const LaunchArgs&, const CUtensorMap*, const CUtensorMap*);
-
-template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
-cudaError_t launch_decode_t(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
-{
-    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG>;
-    auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES, PG>;
-    static int blocks_per_sm = 0;
-    if (blocks_per_sm == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        int occ = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, C::kThreads, C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        blocks_per_sm = occ > 0 ? occ : 1;
-    }
-    const int n_row_tiles = (int)((a.N + C::kRB - 1) / C::kRB);
-    const int n_mblocks = (int)((a.M + C::kMB - 1) / C::kMB);
-    const long long units = (long long)n_row_tiles * a.S * n_mblocks;
-    long long grid = (long long)a.sm_count * blocks_per_sm;
-    if (a.max_blocks > 0 && grid > a.max_blocks) grid = a.max_blocks;
-    if (grid > units) grid = units;
-    const int direct = (a.S == 1);
-
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(C::kThreads);
-    cfg.dynamicSmemBytes = C::kSmemBytes;
-    cfg.stream = a.stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, *map_w, *map_x, a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N,
-                                       (int)a.K, (int)a.seg_len, a.S, direct, n_row_tiles, n_mblocks, a.status);
-    if (e != cudaSuccess) return e;
-    if (!direct) return launch_combine(a);
-    return cudaSuccess;
-}
-
-struct DecodeEntry {
-    DecodeConfig cfg;
-    DecodeLaunchFn fn;
-};
-
-#define DEC(MT, WM, RT, WR, KC, ST, PG) \
-    { {MT, WM, RT, WR, KC, ST, 0}, &launch_decode_t<MT, WM, RT, WR, KC, ST, PG> }
-
-// Tilings per batch class (all produce identical bits).  The first entry of a class is the
-// automatic choice.
-constexpr int kVariantsPerClass = 4;
-const DecodeEntry kTable[6][kVariantsPerClass] = {
-    /* M <= 1  */ {DEC(1, 1, 4, 4, 256, 8, 1), DEC(1, 1, 8, 4, 256, 6, 1), DEC(1, 1, 8, 2, 256, 6, 1), DEC(1, 1, 2, 4, 256, 8, 1)},
-    /* M <= 2  */ {DEC(2, 1, 4, 4, 256, 8, 1), DEC(2, 1, 8, 4, 256, 6, 1), DEC(2, 1, 8, 2, 256, 6, 1), DEC(2, 1, 2, 4, 256, 8, 1)},
-    /* M <= 4  */ {DEC(4, 1, 4, 4, 256, 6, 1), DEC(4, 1, 8, 4, 256, 4, 1), DEC(4, 1, 8, 2, 256, 6, 1), DEC(4, 1, 4, 8, 256, 4, 1)},
-    /* M <= 8  */ {DEC(8, 1, 4, 4, 256, 5, 1), DEC(8, 1, 8, 8, 256, 5, 4), DEC(8, 1, 8, 4, 256, 4, 4), DEC(8, 1, 4, 8, 256, 4, 1)},
-    /* M <= 16 */ {DEC(8, 2, 8, 4, 256, 3, 4), DEC(8, 2, 8, 4, 256, 6, 4), DEC(8, 2, 8, 2, 256, 4, 4), DEC(8, 2, 4, 4, 256, 4, 1)},
-    /* M > 16  */ {DEC(8, 4, 8, 2, 256, 5, 4), DEC(8, 4, 8, 2, 128, 5, 4), DEC(8, 4, 8, 1, 256, 4, 4), DEC(8, 4, 4, 2, 128, 6, 1)},
-};
 
 int m_class(int64_t M) { return M <= 1 ? 0 : M <= 2 ? 1 : M <= 4 ? 2 : M <= 8 ? 3 : M <= 16 ? 4 : 5; }
 
+// Predicted cost of a tiling: the rows of W (padded to whole tiles) that the busiest SM has to
+// process, corrected for how well the tile amortises shared-memory traffic and for having too few
+// warps resident to hide latency.  Heuristic, checked against sweeps on the Llama-3-8B shapes.
+double tiling_cost(const DecodeEntry& e, int64_t M, int64_t N, int S, int sm_count)
+{
+    const DecodeConfig& c = e.cfg;
+    const int occ = e.occupancy();
+    if (occ <= 0) return 1e300;
+    const int64_t rb = (int64_t)c.rt * c.wr, mb = (int64_t)c.mt * c.wm;
+    const int64_t units = ((N + rb - 1) / rb) * S * ((M + mb - 1) / mb);
+    const int64_t per_sm = (units + sm_count - 1) / sm_count;
+    const double rows = (double)per_sm * (double)rb;
+    const int64_t resident = per_sm < occ ? per_sm : occ;
+    const double warps = (double)resident * c.wm * c.wr;
+    const double latency_penalty = warps >= 8.0 ? 1.0 : 8.0 / warps;
+    // shared-memory wavefronts per packed FMA of an (mt x rt) warp tile
+    const double r = (4.0 * c.mt + 2.0 * c.rt) / ((double)c.mt * c.rt);
+    const double weight = M >= 8 ? 0.35 : 0.35 * (double)M / 8.0;
+    return rows * latency_penalty * (1.0 + weight * r);
+}
+
 }  // namespace
 
-int decode_num_variants() { return kVariantsPerClass; }
+int decode_num_variants()
+{
+    int n = 0;
+    for (int c = 0; c < 6; ++c) n = class_table(c)->count > n ? class_table(c)->count : n;
+    return n;
+}
 
 bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfig* out)
 {
-    (void)N; (void)K;
-    if (variant < 0 || variant > kVariantsPerClass) return false;
+    (void)K;
     const int cls = m_class(M);
-    const int v = variant == 0 ? 0 : variant - 1;
-    *out = kTable[cls][v].cfg;
-    out->id = cls * kVariantsPerClass + v;
+    const DecodeClassTable* t = class_table(cls);
+    if (variant < 0 || variant > t->count) return false;
+    int pick = variant - 1;
+    if (variant == 0) {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+        // the split factor does not depend on the tiling; recompute it from the shape
+        det_linear_params_t prm;
+        const int S = fill_params(M, N, K, &prm) == DET_OK ? prm.S : 1;
+        double best = 1e301;
+        pick = 0;
+        for (int i = 0; i < t->count; ++i) {
+            const double c = tiling_cost(t->entries[i], M, N, S, sms);
+            if (c < best) { best = c; pick = i; }
+        }
+    }
+    *out = t->entries[pick].cfg;
+    out->id = cls * 64 + pick;
     return true;
 }
 
@@ -462,7 +79,7 @@ cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const C
 {
     DecodeConfig cfg;
     if (!decode_config_for(a.M, a.N, a.K, a.variant, &cfg)) return cudaErrorInvalidValue;
-    return kTable[cfg.id / kVariantsPerClass][cfg.id % kVariantsPerClass].fn(a, map_w, map_x);
+    return class_table(cfg.id / 64)->entries[cfg.id % 64].fn(a, map_w, map_x);
 }
 
 }  // namespace detlin

@@ -7,8 +7,9 @@
 
 namespace detlin {
 
-// Decode order (V=4, L=32, P=2): one warp per (row n, segment s); lane l owns k = c + 4l + j in every
-// 128-element chunk and feeds sub-chain j & 1; leaves are summed adjacent-first.
+// Decode order (V=4, L=32, P=1): one warp per (row n, segment s); lane l owns k = c + 4l + j in every
+// 128-element chunk and accumulates them in ascending order into one chain; the 32 lanes are summed
+// adjacent-first.
 __global__ void __launch_bounds__(256)
 generic_decode_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, const float* __restrict__ b,
                       float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct)
@@ -23,21 +24,16 @@ generic_decode_kernel(const float* __restrict__ x, const uint16_t* __restrict__ 
     const uint16_t* wrow = W + n * K;
     for (int64_t m = 0; m < M; ++m) {
         const float* xrow = x + m * K;
-        float a0 = 0.0f, a1 = 0.0f;
+        float a = 0.0f;
         for (int64_t c = k_lo; c < k_hi; c += 128) {
             const int64_t k0 = c + 4 * lane;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int64_t k = k0 + j;
-                if (k < k_hi) {
-                    const float xv = xrow[k];
-                    const float wv = up_bf16(wrow[k]);
-                    if (j & 1) a1 = __fmaf_rn(xv, wv, a1);
-                    else       a0 = __fmaf_rn(xv, wv, a0);
-                }
+                if (k < k_hi) a = __fmaf_rn(xrow[k], up_bf16(wrow[k]), a);
             }
         }
-        float t = lane_tree_sum(__fadd_rn(a0, a1));
+        const float t = lane_tree_sum(a);
         if (lane == 0) {
             if (direct) out[m * N + n] = b ? __fadd_rn(t, b[n]) : t;
             else        out[((int64_t)s * M + m) * N + n] = t;

@@ -40,7 +40,7 @@ det_status_t fill_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* o
     }
     det_linear_params_t p{};
     p.M = M; p.N = N; p.K = K;
-    if (M <= kDecodeMaxM) { p.bucket = 0; p.V = 4; p.L = 32; p.P = 2; }
+    if (M <= kDecodeMaxM) { p.bucket = 0; p.V = 4; p.L = 32; p.P = 1; }
     else                  { p.bucket = 1; p.V = 2; p.L = 1;  p.P = 2; }
     const int64_t s_req = split_request(M, N, K);
     const int64_t n_gran = ceil_div(K, kSegmentGranule);
