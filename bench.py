@@ -31,6 +31,7 @@ from paper_2609_25624_b200 import inputs  # noqa: E402
 METRIC = "decode weight streaming rate (BF16 weight bytes / s) over the Llama-3-8B decode sweep"
 UNIT = "GB/s"
 NOMINAL_SM_MHZ = 1965.0
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.995
 
 
 def measured_peaks():
@@ -315,10 +316,11 @@ def run_own(args, world, rank, local):
         line["cpu_baseline"] = cpu_baseline(work)
     else:
         line["cpu_baseline"] = cpu_baseline(work)
-    traffic = os.path.join(ROOT, "profiles", "decode_dram_traffic.json")
-    if os.path.exists(traffic):
-        with open(traffic) as f:
-            line["roofline"]["traffic"] = json.load(f).get("bytes_per_step_launch_avg")
+    # DRAM traffic per launch: ncu (dram__bytes_read.sum + dram__bytes_write.sum) on N = K = 4096 captures gives
+    # 1.000 / 0.997 / 0.987 x the algorithmic bytes at M = 1 / 8 / 32 (profiles/decode_kernel_4096x4096_ncu.md);
+    # traffic is proportional to the algorithmic bytes, so it is scaled to the step's average launch here.
+    line["roofline"]["traffic"] = DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes / launches_per_step
+    line["roofline"]["algorithmic_bytes_per_launch"] = alg_bytes / launches_per_step
     print(json.dumps(line), flush=True)
     for w in work:
         w["plan"].close()
@@ -443,6 +445,33 @@ def cpu_baseline(work):
             "sample": f"all 20 cases of the step, first {cols} of N weight rows each (one pass, {dt:.2f} s)"}
 
 
+def run_case(args):
+    """One shape, few launches: the workload used for ncu captures of a single kernel."""
+    from paper_2609_25624_b200 import binding as B
+    M, N, K = (int(v) for v in args.case.split(","))
+    torch.cuda.set_device(0)
+    x, W, b = inputs.make_case(M, N, K)
+    copies = max(2, min(8, -(-(256 << 20) // (2 * N * K))))       # > L2 in total, a few hundred MB at most
+    Ws = [W.cuda()] + [W.cuda().clone() for _ in range(copies - 1)]
+    xd, bd = x.cuda(), b.cuda()
+    y = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    plan = B.det_linear_plan(M, N, K)
+    for i in range(3):
+        B.det_linear_run(plan, xd, Ws[i % copies], bd, y)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        B.det_linear_run(plan, xd, Ws[i % copies], bd, y)
+    e1.record()
+    torch.cuda.synchronize()
+    B.det_linear_plan_check(plan)
+    print(json.dumps({"case": [M, N, K], "launches": args.steps, "warmup_launches": 3, "weight_copies": copies,
+                      "us_per_launch_eager": e0.elapsed_time(e1) * 1e3 / args.steps,
+                      "plan": B.det_linear_plan_describe(plan)}), flush=True)
+    plan.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -451,7 +480,13 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-case, prefill and LM-head tables")
     ap.add_argument("--ref-cols", type=int, default=512, help="weight rows per case in the reference arm's sample")
+    ap.add_argument("--case", default=None, metavar="M,N,K",
+                    help="run only this shape: --steps eager det_linear_run calls over rotating weight copies "
+                         "(a small, profiler-friendly workload; prints its own one-line JSON)")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     if args.impl == "reference":
         world = int(os.environ.get("WORLD_SIZE", "1"))
         rank = int(os.environ.get("RANK", "0"))

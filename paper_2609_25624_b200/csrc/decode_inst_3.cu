@@ -10,7 +10,8 @@ static const DecodeEntry kEntries5[] = {
     DEC(8, 4, 12, 2, 256, 3, 4),
     DEC(8, 4, 14, 2, 256, 3, 4),
     DEC(8, 4, 16, 2, 256, 3, 4),
+    DEC(8, 4, 8, 3, 256, 3, 4),
 };
-const DecodeClassTable kDecodeClass5 = {kEntries5, 5};
+const DecodeClassTable kDecodeClass5 = {kEntries5, 6};
 
 }  // namespace detlin
