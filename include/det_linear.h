@@ -11,7 +11,7 @@
  *
  * Reduction order, version 1 (what "the same bits" means):
  *   bucket   = decode if M <= 64, else prefill                                  (R2, R4)
- *   decode : V = 4, L = 32, P = 1        prefill: V = 2, L = 1, P = 2
+ *   decode : V = 4, L = 32, P = 1        prefill: V = 1, L = 1, P = 1 (strictly ascending k)
  *   K is cut into S contiguous segments of seg_len elements (a multiple of 256; only the last
  *   may be short); S is shape-pure and, for decode, independent of M               (R3, R4)
  *   inside a segment, chunks of V*L elements are walked in ascending k; "lane" l owns the V

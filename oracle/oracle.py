@@ -28,24 +28,39 @@ def _ceil_div(a: int, b: int) -> int:
     return -(-a // b)
 
 
+def _segments_for(K: int, s_req: int):
+    """Segment layout for a requested split: boundaries on multiples of the granule, every segment
+    non-empty.  Returns (seg_len, S)."""
+    n_gran = _ceil_div(K, SEGMENT_GRANULE)
+    gran_per_seg = _ceil_div(n_gran, min(s_req, n_gran))
+    return SEGMENT_GRANULE * gran_per_seg, _ceil_div(n_gran, gran_per_seg)
+
+
 def split_request(M: int, N: int, K: int) -> int:
     """Requested number of K segments before clamping to what K allows.
 
     Decode (never reads M, rule R4): 1 when N >= 4096 (enough rows to fill the machine, like the
     paper's lm_head "prefers no split"); otherwise the smallest power of two with N*S >= 4096.
-    Prefill: the smallest power of two S <= 16 with tiles*S >= 1024 where tiles counts 128x128
-    output tiles, never cutting a segment below 512 elements.
-    """
+    Prefill: the request in 1..16 that minimises rounds * (seg_len + overhead) * occupancy_factor,
+    with tiles = number of 128x128 output tiles, units = tiles * S, rounds = ceil(units / 148),
+    overhead = 8 k-steps per work unit plus 32 when partials are written and combined,
+    occupancy_factor = 9 if units <= 148 else 8; ties go to the larger request.  The constants are
+    frozen parts of the order definition (tuned once on a 148-SM part, never read from the device)."""
     if M <= DECODE_MAX_M:
         s = 1
         while N * s < 4096:
             s *= 2
         return s
     tiles = _ceil_div(M, 128) * _ceil_div(N, 128)
-    s = 1
-    while s < 16 and tiles * s < 1024 and K // (2 * s) >= 512:
-        s *= 2
-    return s
+    best, best_cost = 1, None
+    for s_req in range(1, 17):
+        seg_len, S = _segments_for(K, s_req)
+        units = tiles * S
+        rounds = _ceil_div(units, 148)
+        cost = rounds * (seg_len + (40 if S > 1 else 8)) * (9 if units <= 148 else 8)
+        if best_cost is None or cost <= best_cost:
+            best, best_cost = s_req, cost
+    return best
 
 
 def order_params(M: int, N: int, K: int) -> dict:
@@ -55,12 +70,8 @@ def order_params(M: int, N: int, K: int) -> dict:
     if M <= DECODE_MAX_M:
         bucket, V, L, P = "decode", 4, 32, 1
     else:
-        bucket, V, L, P = "prefill", 2, 1, 2
-    s_req = split_request(M, N, K)
-    n_gran = _ceil_div(K, SEGMENT_GRANULE)
-    gran_per_seg = _ceil_div(n_gran, min(s_req, n_gran))
-    seg_len = SEGMENT_GRANULE * gran_per_seg
-    S = _ceil_div(n_gran, gran_per_seg)
+        bucket, V, L, P = "prefill", 1, 1, 1
+    seg_len, S = _segments_for(K, split_request(M, N, K))
     return {"bucket": bucket, "V": V, "L": L, "P": P, "seg_len": seg_len, "S": S,
             "order_version": ORDER_VERSION}
 

@@ -41,8 +41,7 @@ generic_decode_kernel(const float* __restrict__ x, const uint16_t* __restrict__ 
     }
 }
 
-// Prefill order (V=2, L=1, P=2): one thread per (m, n, segment): an even-k chain and an odd-k chain,
-// added once at the end of the segment.
+// Prefill order (V=1, L=1, P=1): one thread per (m, n, segment), one chain, strictly ascending k.
 __global__ void __launch_bounds__(256)
 generic_prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, const float* __restrict__ b,
                        float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct)
@@ -55,12 +54,8 @@ generic_prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__
     const int64_t k_hi = (k_lo + seg_len < K) ? k_lo + seg_len : K;
     const float* xrow = x + m * K;
     const uint16_t* wrow = W + n * K;
-    float a0 = 0.0f, a1 = 0.0f;
-    for (int64_t k = k_lo; k < k_hi; k += 2) {
-        a0 = __fmaf_rn(xrow[k], up_bf16(wrow[k]), a0);
-        if (k + 1 < k_hi) a1 = __fmaf_rn(xrow[k + 1], up_bf16(wrow[k + 1]), a1);
-    }
-    const float t = __fadd_rn(a0, a1);
+    float t = 0.0f;
+    for (int64_t k = k_lo; k < k_hi; ++k) t = __fmaf_rn(xrow[k], up_bf16(wrow[k]), t);
     if (direct) out[m * N + n] = b ? __fadd_rn(t, b[n]) : t;
     else        out[((int64_t)s * M + m) * N + n] = t;
 }

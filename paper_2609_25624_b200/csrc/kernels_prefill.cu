@@ -1,15 +1,20 @@
 // Prefill kernel (bucket M > 64): register-tiled FP32 GEMM on the CUDA cores (rule R1: IEEE FMA only,
-// never tensor cores) in the frozen prefill order (V=2, L=1, P=2): every output keeps two
-// accumulation chains per K segment, one over the even k and one over the odd k, each strictly
-// ascending; they are added once at the end of the segment, segments are summed in ascending order
-// and the bias comes last.  The two chains of an output are exactly the two halves of one packed
-// FP32x2 accumulator, so one fma.rn.f32x2 advances both chains by one element each, with the
-// operands (x[m,k], x[m,k+1]) and (up(W[n,k]), up(W[n,k+1])) taken as they lie in memory.
+// never tensor cores) in the frozen prefill order (V=1, L=1, P=1): every output is one accumulation
+// chain per K segment, strictly ascending in k (the order of the paper's own kernels, supplement C on
+// rule R2); segments are summed in ascending order and the bias comes last.
+//
+// One packed fma.rn.f32x2 advances the chains of two neighbouring output columns (n, n+1) of the
+// same row m by one element: operands (x[m,k], x[m,k]) and (up(W[n,k]), up(W[n+1,k])), accumulator
+// (acc[m,n], acc[m,n+1]).  Each half is an ordinary fma.rn.f32, so the pairing is invisible in the
+// bits.  Measured on B200 this loop sustains more than the scalar-FMA form of the same tile because
+// the packed instruction leaves every other issue slot free for the shared-memory loads.
 //
 // Schedule (numerically inert): 128 x 128 output tile per block, 256 threads, 8 x 8 outputs per
-// thread, K walked in slabs of 32.  BF16 weights are widened to FP32 once per block while the slab
-// is staged into shared memory (so HBM and L2 only ever carry BF16 weights, Eq. 2), activations are
-// staged as they are.  Global loads of slab i+1 are in flight while slab i is multiplied.
+// thread (4 column pairs), two blocks per SM, K walked in slabs of 32 with two slab buffers.  Both
+// operands are staged k-major ([k][m] and [k][n]) so that a thread reads its eight x values and its
+// eight weights of one k with four 16-byte loads.  BF16 weights are widened to FP32 once per block
+// while the slab is staged (HBM and L2 only ever carry BF16 weights, Eq. 2).  Global loads of slab
+// i+1 are in flight while slab i is multiplied.
 #include "internal.h"
 #include "device_utils.cuh"
 
@@ -19,10 +24,9 @@ namespace {
 
 constexpr int BM = 128, BN = 128, BK = 32;
 constexpr int kThreads = 256;
-constexpr int kPitch = 129;                        // 16-byte chunks per k-quad row (odd: conflict-free staging)
-constexpr int kQuads = BK / 4;                     // k-quads per slab
-constexpr int kTileChunks = kQuads * kPitch;       // 16-byte chunks per operand tile
-constexpr int kSmemBytes = 2 /*buffers*/ * 2 /*operands*/ * kTileChunks * 16;
+constexpr int kPitch = 132;                         // floats per k row: 128 + 4 keeps 16-byte alignment
+constexpr int kTileFloats = BK * kPitch;
+constexpr int kSmemBytes = 2 /*buffers*/ * 2 /*operands*/ * kTileFloats * 4;
 
 __device__ __forceinline__ float4 lds128(uint32_t addr)
 {
@@ -30,9 +34,9 @@ __device__ __forceinline__ float4 lds128(uint32_t addr)
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ void sts128(uint32_t addr, float4 v)
+__device__ __forceinline__ void sts32(uint32_t addr, float v)
 {
-    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 __device__ __forceinline__ uint4 ldg128_nc(const void* p)
 {
@@ -41,14 +45,14 @@ __device__ __forceinline__ uint4 ldg128_nc(const void* p)
     return v;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, const float* __restrict__ bias,
                float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct, int tiles_m, int tiles_n)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t smem = (uint32_t)__cvta_generic_to_shared(smem_raw);
-    // buffer b: x tile at smem + b*2*T, w tile at smem + (b*2+1)*T, T = kTileChunks*16 bytes
-    constexpr uint32_t T = kTileChunks * 16;
+    // buffer b: x tile at smem + b*2*T, w tile at smem + (b*2+1)*T, T = kTileFloats*4 bytes
+    constexpr uint32_t T = kTileFloats * 4;
 
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
@@ -63,72 +67,90 @@ prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, cons
     const int k_lo = s * seg_len;
     const int k_hi = min(K, k_lo + seg_len);
 
-    // ---- staging assignment ----
-    // x tile: 128 rows x 8 quads = 1024 chunks, 4 per thread: chunk p = tid + 256 j -> row p / 8, quad p % 8
-    // w tile: 128 rows x 4 octets (8 BF16 = 16 bytes) = 512 pieces, 2 per thread: p = tid + 256 j -> row p / 4, octet p % 4
+    // ---- staging assignment (global rows are k-contiguous, shared tiles are k-major: a transpose) ----
+    // x tile: 128 rows x 8 quads (4 floats = 16 bytes).  Piece p = tid + 256 j: half o = p & 1,
+    //   row r = (p >> 1) & 127, quad q = 2 * (p >> 8) + o.  Two neighbouring lanes read one 32-byte
+    //   sector; the four scalar stores of a lane go to k rows 4q .. 4q+3, conflict-free across the warp
+    //   (bank = 16 o + 4 e + r mod 32 over 16 consecutive r and o in {0, 1}).
+    // w tile: 128 rows x 4 octets (8 BF16 = 16 bytes).  Piece p = tid + 256 j: half o = p & 1,
+    //   row r = (p >> 1) & 127, octet c = 2 * (p >> 8) + o; eight scalar stores to k rows 8c .. 8c+7
+    //   (two-way bank conflicts between the two halves; 16 stores per thread and slab).
     const float* xg[4];
     uint32_t xs_off[4];
+    int xk[4];
     bool xok[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int p = tid + 256 * j;
-        const int r = p >> 3, q = p & 7;
+        const int o = p & 1, r = (p >> 1) & 127, q = 2 * (p >> 8) + o;
         const int m = m0 + r;
         xok[j] = m < M;
+        xk[j] = q * 4;
         xg[j] = x + (long long)(xok[j] ? m : 0) * K + q * 4;
-        xs_off[j] = (uint32_t)(q * kPitch + r) * 16;
+        xs_off[j] = (uint32_t)((q * 4) * kPitch + r) * 4;
     }
     const uint16_t* wg[2];
     uint32_t ws_off[2];
+    int wk[2];
     bool wok[2];
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
         const int p = tid + 256 * j;
-        const int r = p >> 2, o = p & 3;
+        const int o = p & 1, r = (p >> 1) & 127, c = 2 * (p >> 8) + o;
         const int n = n0 + r;
         wok[j] = n < N;
-        wg[j] = W + (long long)(wok[j] ? n : 0) * K + o * 8;
-        ws_off[j] = (uint32_t)((2 * o) * kPitch + r) * 16;
+        wk[j] = c * 8;
+        wg[j] = W + (long long)(wok[j] ? n : 0) * K + c * 8;
+        ws_off[j] = (uint32_t)((c * 8) * kPitch + r) * 4;
     }
 
-    float4 xr[4];
+    uint4 xr[4];
     uint4 wr[2];
     auto load_slab = [&](int k0) {
         // K % 8 == 0: an octet of weights / a quad of activations is entirely inside or outside [.., k_hi)
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = (tid + 256 * j) & 7;
-            if (xok[j] && k0 + q * 4 < k_hi) {
-                const uint4 t = ldg128_nc(xg[j] + k0);
-                xr[j] = make_float4(__uint_as_float(t.x), __uint_as_float(t.y), __uint_as_float(t.z), __uint_as_float(t.w));
-            } else {
-                xr[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            if (xok[j] && k0 + xk[j] < k_hi) xr[j] = ldg128_nc(xg[j] + k0);
+            else xr[j] = make_uint4(0u, 0u, 0u, 0u);
         }
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-            const int o = (tid + 256 * j) & 3;
-            if (wok[j] && k0 + o * 8 < k_hi) wr[j] = ldg128_nc(wg[j] + k0);
+            if (wok[j] && k0 + wk[j] < k_hi) wr[j] = ldg128_nc(wg[j] + k0);
             else wr[j] = make_uint4(0u, 0u, 0u, 0u);
         }
     };
     auto store_slab = [&](int buf) {
         const uint32_t xb = smem + (uint32_t)(buf * 2) * T, wb = xb + T;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) sts128(xb + xs_off[j], xr[j]);
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t a = xb + xs_off[j];
+            sts32(a, __uint_as_float(xr[j].x));
+            sts32(a + kPitch * 4, __uint_as_float(xr[j].y));
+            sts32(a + 2 * kPitch * 4, __uint_as_float(xr[j].z));
+            sts32(a + 3 * kPitch * 4, __uint_as_float(xr[j].w));
+        }
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-            // widen the eight BF16 weights to FP32 (exact): quad 2o holds k..k+3, quad 2o+1 holds k+4..k+7
-            sts128(wb + ws_off[j], make_float4(up_lo(wr[j].x), up_hi(wr[j].x), up_lo(wr[j].y), up_hi(wr[j].y)));
-            sts128(wb + ws_off[j] + kPitch * 16, make_float4(up_lo(wr[j].z), up_hi(wr[j].z), up_lo(wr[j].w), up_hi(wr[j].w)));
+            // widen the eight BF16 weights to FP32 (exact) on the way to shared memory
+            const uint32_t a = wb + ws_off[j];
+            sts32(a, up_lo(wr[j].x));
+            sts32(a + kPitch * 4, up_hi(wr[j].x));
+            sts32(a + 2 * kPitch * 4, up_lo(wr[j].y));
+            sts32(a + 3 * kPitch * 4, up_hi(wr[j].y));
+            sts32(a + 4 * kPitch * 4, up_lo(wr[j].z));
+            sts32(a + 5 * kPitch * 4, up_hi(wr[j].z));
+            sts32(a + 6 * kPitch * 4, up_lo(wr[j].w));
+            sts32(a + 7 * kPitch * 4, up_hi(wr[j].w));
         }
     };
 
-    float2 acc[8][8];        // [i][j] -> output (m0 + ty + 16 i, n0 + tx + 16 j): (even-k chain, odd-k chain)
+    // acc[i][j]: rows m0 + (i < 4 ? 4 ty + i : 64 + 4 ty + i - 4); column pair j:
+    //   (n0 + 4 tx + 2 j, +1) for j < 2, (n0 + 64 + 4 tx + 2 (j - 2), +1) for j >= 2
+    float2 acc[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
+        for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
 
     load_slab(k_lo);
     store_slab(0);
@@ -138,28 +160,24 @@ prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, cons
     for (int k0 = k_lo; k0 < k_hi; k0 += BK) {
         const bool more = k0 + BK < k_hi;
         if (more) load_slab(k0 + BK);
-        const uint32_t xb = smem + (uint32_t)(buf * 2) * T + (uint32_t)ty * 16;
-        const uint32_t wb = smem + (uint32_t)(buf * 2 + 1) * T + (uint32_t)tx * 16;
-        // k beyond the end of the segment is skipped, not zero-filled: only whole valid quads run
-        const int nq = min(kQuads, (k_hi - k0) >> 2);
-#pragma unroll 2
-        for (int q = 0; q < nq; ++q) {
-            float4 xf[8], wf[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) xf[i] = lds128(xb + (uint32_t)(q * kPitch + 16 * i) * 16);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) wf[j] = lds128(wb + (uint32_t)(q * kPitch + 16 * j) * 16);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float2 xa = make_float2(xf[i].x, xf[i].y);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = __ffma2_rn(xa, make_float2(wf[j].x, wf[j].y), acc[i][j]);
-            }
+        const uint32_t xb = smem + (uint32_t)(buf * 2) * T + (uint32_t)(ty * 4) * 4;
+        const uint32_t wb = smem + (uint32_t)(buf * 2 + 1) * T + (uint32_t)(tx * 4) * 4;
+        // k beyond the end of the segment is skipped, not zero-filled
+        const int nk = min(BK, k_hi - k0);
+#pragma unroll 4
+        for (int kk = 0; kk < nk; ++kk) {
+            const float4 xa = lds128(xb + (uint32_t)(kk * kPitch) * 4);
+            const float4 xc = lds128(xb + (uint32_t)(kk * kPitch + 64) * 4);
+            const float4 wa = lds128(wb + (uint32_t)(kk * kPitch) * 4);
+            const float4 wc = lds128(wb + (uint32_t)(kk * kPitch + 64) * 4);
+            const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xc.x, xc.y, xc.z, xc.w};
+            const float2 wp[4] = {make_float2(wa.x, wa.y), make_float2(wa.z, wa.w), make_float2(wc.x, wc.y),
+                                  make_float2(wc.z, wc.w)};
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const float2 xc = make_float2(xf[i].z, xf[i].w);
+                const float2 x2 = make_float2(xv[i], xv[i]);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = __ffma2_rn(xc, make_float2(wf[j].z, wf[j].w), acc[i][j]);
+                for (int j = 0; j < 4; ++j) acc[i][j] = __ffma2_rn(x2, wp[j], acc[i][j]);
             }
         }
         if (more) store_slab(buf ^ 1);
@@ -167,21 +185,28 @@ prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, cons
         buf ^= 1;
     }
 
-    // ---- epilogue: even + odd chain, then bias (direct) or the segment's partial ----
+    // ---- epilogue: bias (direct) or the segment's partial ----
+    const bool vec_ok = (N % 4 == 0);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const int m = m0 + ty + 16 * i;
+        const int m = m0 + (i < 4 ? 4 * ty + i : 64 + 4 * ty + (i - 4));
         if (m >= M) continue;
+        float* orow = direct ? out + (long long)m * N : out + ((long long)s * M + m) * N;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int n = n0 + tx + 16 * j;
-            if (n >= N) continue;
-            float t = __fadd_rn(acc[i][j].x, acc[i][j].y);
-            if (direct) {
-                if (bias) t = __fadd_rn(t, bias[n]);
-                out[(long long)m * N + n] = t;
+        for (int h = 0; h < 2; ++h) {
+            const int n = n0 + 64 * h + 4 * tx;
+            float v[4] = {acc[i][2 * h].x, acc[i][2 * h].y, acc[i][2 * h + 1].x, acc[i][2 * h + 1].y};
+            if (direct && bias) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (n + e < N) v[e] = __fadd_rn(v[e], bias[n + e]);
+            }
+            if (vec_ok && n + 3 < N) {
+                *reinterpret_cast<float4*>(orow + n) = make_float4(v[0], v[1], v[2], v[3]);
             } else {
-                out[((long long)s * M + m) * N + n] = t;
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (n + e < N) orow[n + e] = v[e];
             }
         }
     }

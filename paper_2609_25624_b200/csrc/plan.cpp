@@ -7,23 +7,46 @@ namespace detlin {
 
 static int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+// Segment layout for a requested split: boundaries on multiples of the granule, every segment
+// non-empty.
+static void segments_for(int64_t K, int64_t s_req, int64_t* seg_len, int64_t* S)
+{
+    const int64_t n_gran = ceil_div(K, kSegmentGranule);
+    const int64_t per_seg = ceil_div(n_gran, s_req < n_gran ? s_req : n_gran);
+    *seg_len = per_seg * kSegmentGranule;
+    *S = ceil_div(n_gran, per_seg);
+}
+
 // Requested split factor before clamping to what K allows.
 //  decode : no split once N alone provides 4096 rows of parallel work (like the paper's lm_head,
 //           which "prefers no split"); below that the smallest power of two with N*S >= 4096.
-//           Never reads M.
-//  prefill: the smallest power of two S <= 16 that yields at least 1024 (128x128 tile, segment)
-//           work units, while keeping segments at least 512 elements long.  The constants were
-//           tuned once for a 148-SM part and are frozen; the SM count is never read.
+//           Never reads M (rule R4).
+//  prefill: the request in 1..16 that minimises  rounds * (seg_len + overhead) * occupancy_factor
+//           where tiles counts 128x128 output tiles, units = tiles * S, rounds = ceil(units / 148),
+//           overhead = 8 k-steps per work unit plus 32 when partials have to be written and combined,
+//           and occupancy_factor = 9 when units <= 148 (one block per SM) else 8; ties go to the
+//           larger split.  148 and the overheads were measured once on a B200 and are frozen
+//           constants of the order definition: the rule is a pure function of (M, N, K) and never
+//           reads the device (rule R2: "tuned once offline and pinned").
 static int split_request(int64_t M, int64_t N, int64_t K)
 {
-    int s = 1;
     if (M <= kDecodeMaxM) {
+        int s = 1;
         while (N * s < 4096) s *= 2;
         return s;
     }
     const int64_t tiles = ceil_div(M, 128) * ceil_div(N, 128);
-    while (s < 16 && tiles * s < 1024 && K / (2 * s) >= 512) s *= 2;
-    return s;
+    int best = 1;
+    int64_t best_cost = -1;
+    for (int s_req = 1; s_req <= 16; ++s_req) {
+        int64_t seg_len, S;
+        segments_for(K, s_req, &seg_len, &S);
+        const int64_t units = tiles * S;
+        const int64_t rounds = ceil_div(units, 148);
+        const int64_t cost = rounds * (seg_len + (S > 1 ? 40 : 8)) * (units <= 148 ? 9 : 8);
+        if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = s_req; }
+    }
+    return best;
 }
 
 det_status_t fill_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* out)
@@ -41,12 +64,11 @@ det_status_t fill_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* o
     det_linear_params_t p{};
     p.M = M; p.N = N; p.K = K;
     if (M <= kDecodeMaxM) { p.bucket = 0; p.V = 4; p.L = 32; p.P = 1; }
-    else                  { p.bucket = 1; p.V = 2; p.L = 1;  p.P = 2; }
-    const int64_t s_req = split_request(M, N, K);
-    const int64_t n_gran = ceil_div(K, kSegmentGranule);
-    const int64_t per_seg = ceil_div(n_gran, s_req < n_gran ? s_req : n_gran);
-    p.seg_len = per_seg * kSegmentGranule;
-    p.S = (int32_t)ceil_div(n_gran, per_seg);
+    else                  { p.bucket = 1; p.V = 1; p.L = 1;  p.P = 1; }
+    int64_t seg_len, S;
+    segments_for(K, split_request(M, N, K), &seg_len, &S);
+    p.seg_len = seg_len;
+    p.S = (int32_t)S;
     p.order_version = kOrderVersion;
     p.kernel = (K % 8 == 0) ? (p.bucket == 0 ? kKernelDecode : kKernelPrefill) : kKernelGeneric;
     p.workspace_bytes = p.S > 1 ? (uint64_t)4 * (uint64_t)p.S * (uint64_t)M * (uint64_t)N : 0;
