@@ -314,6 +314,10 @@ def run_own(args, world, rank, local):
         line["prefill"] = prefill_table(B, dev, st, fp32_peak)
         line["lm_head"] = lm_head_table(B, dev, st, hbm_peak, fp32_peak)
         line["cpu_baseline"] = cpu_baseline(work)
+        for w in work:                       # free the sweep's 2.2 GB before the 15 GB stack
+            w["plan"].close()
+        work.clear()
+        line["stack"] = stack_table(dev, st, hbm_peak)
     else:
         line["cpu_baseline"] = cpu_baseline(work)
     # DRAM traffic per launch: ncu (dram__bytes_read.sum + dram__bytes_write.sum) on N = K = 4096 captures gives
@@ -324,6 +328,27 @@ def run_own(args, world, rank, local):
     print(json.dumps(line), flush=True)
     for w in work:
         w["plan"].close()
+
+
+def stack_table(dev, st, hbm_peak):
+    """Full decode-step linear stack (32 layers x 4 projections + LM head + argmax, 15 GB of BF16
+    weights drawn on the device): one CUDA graph per step, 16 timed steps, batch 1 and 8."""
+    from paper_2609_25624_b200.stack import LinearStack, initial_activations
+    stack = LinearStack(n_layers=32, device=dev)
+    stack.load_device_random(seed=0)
+    wbytes = sum(2 * w.numel() for layer in stack.weights for w in layer.values()) + 2 * stack.lm_head.numel()
+    rows = []
+    for M in (1, 8):
+        plans = stack.plans(M)
+        x = initial_activations(M).to(dev)
+        with torch.cuda.stream(st):
+            stack.step(plans, x)
+            torch.cuda.synchronize()
+        ms = time_graph(lambda: stack.step(plans, x), 16, st)
+        rows.append({"M": M, "ms_per_step": ms, "weight_gbs": wbytes / ms / 1e6, "pct_hbm": 100 * wbytes / ms / 1e6 / hbm_peak,
+                     "tokens_per_s": 1e3 * M / ms})
+    stack.close()
+    return {"weight_bytes": wbytes, "kernels_per_step": 32 * 4 + 2, "cases": rows}
 
 
 def calibration(B, dev, fp32_peak):
