@@ -328,37 +328,42 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                 if (!mbar_wait(full0 + 8 * st, (it / STAGES) & 1, abort_flag, status, 2)) { ok = false; break; }
                 const uint32_t xs = smem_base + st * C::kStageBytes + (wm * MT) * (KC * 4) + lane * 16;
                 const uint32_t ws = smem_base + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * 8;
-#pragma unroll(MT * RT >= 64 ? 1 : 2)
-                for (int cc = 0; cc < KC / 128; ++cc) {
-                    // Elements beyond the end of K are skipped, not zero-filled (K % 4 == 0 here, so a
-                    // lane's four elements are all inside or all outside).  Whole chunks take the
-                    // warp-uniform branch.
-                    const int kc0 = k0 + cc * 128;
-                    if (kc0 + 128 <= un.k_hi || kc0 + 4 * lane < un.k_hi) {
-                        uint2 w[RT];
-                        float4 xv[MT];
+                // One 128-element chunk: the lane's four elements of every row / batch row of the warp tile.
+                auto chunk = [&](int cc) {
+                    uint2 w[RT];
+                    float4 xv[MT];
 #pragma unroll
-                        for (int q = 0; q < RT; ++q) w[q] = lds64(ws + q * (KC * 2) + cc * 256);
+                    for (int q = 0; q < RT; ++q) w[q] = lds64(ws + q * (KC * 2) + cc * 256);
 #pragma unroll
-                        for (int m = 0; m < MT; ++m) xv[m] = lds128(xs + m * (KC * 4) + cc * 512);
+                    for (int m = 0; m < MT; ++m) xv[m] = lds128(xs + m * (KC * 4) + cc * 512);
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {          // the lane's four elements, ascending
-                            float2 wp[RT / 2];
+                    for (int kk = 0; kk < 4; ++kk) {          // the lane's four elements, ascending
+                        float2 wp[RT / 2];
 #pragma unroll
-                            for (int j = 0; j < RT / 2; ++j) {
-                                const uint32_t wa = (kk < 2) ? w[2 * j].x : w[2 * j].y;
-                                const uint32_t wb = (kk < 2) ? w[2 * j + 1].x : w[2 * j + 1].y;
-                                wp[j] = (kk & 1) ? make_float2(up_hi(wa), up_hi(wb)) : make_float2(up_lo(wa), up_lo(wb));
-                            }
+                        for (int j = 0; j < RT / 2; ++j) {
+                            const uint32_t wa = (kk < 2) ? w[2 * j].x : w[2 * j].y;
+                            const uint32_t wb = (kk < 2) ? w[2 * j + 1].x : w[2 * j + 1].y;
+                            wp[j] = (kk & 1) ? make_float2(up_hi(wa), up_hi(wb)) : make_float2(up_lo(wa), up_lo(wb));
+                        }
 #pragma unroll
-                            for (int m = 0; m < MT; ++m) {
-                                const float xk = kk == 0 ? xv[m].x : kk == 1 ? xv[m].y : kk == 2 ? xv[m].z : xv[m].w;
-                                const float2 x2 = make_float2(xk, xk);
+                        for (int m = 0; m < MT; ++m) {
+                            const float xk = kk == 0 ? xv[m].x : kk == 1 ? xv[m].y : kk == 2 ? xv[m].z : xv[m].w;
+                            const float2 x2 = make_float2(xk, xk);
 #pragma unroll
-                                for (int j = 0; j < RT / 2; ++j) acc[m][j] = __ffma2_rn(x2, wp[j], acc[m][j]);
-                            }
+                            for (int j = 0; j < RT / 2; ++j) acc[m][j] = __ffma2_rn(x2, wp[j], acc[m][j]);
                         }
                     }
+                };
+                if (k0 + KC <= un.k_hi) {
+                    // whole stage inside the segment: no per-lane test
+#pragma unroll(MT * RT >= 64 ? 1 : 2)
+                    for (int cc = 0; cc < KC / 128; ++cc) chunk(cc);
+                } else {
+                    // Last stage of a ragged K: elements beyond the end are skipped, not zero-filled
+                    // (K % 4 == 0 here, so a lane's four elements are all inside or all outside).
+#pragma unroll 1
+                    for (int cc = 0; cc < KC / 128; ++cc)
+                        if (k0 + cc * 128 + 4 * lane < un.k_hi) chunk(cc);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * st);
