@@ -379,11 +379,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                     v[m * RT + 2 * j] = acc[m][j].x;
                     v[m * RT + 2 * j + 1] = acc[m][j].y;
                 }
-            lane_tree_scatter<MT * RT>(v, lane);
             constexpr int NV = MT * RT;
             constexpr int kKeep = Scatter<NV>::kKeep;
             constexpr int kSteps = Scatter<NV>::kSteps;
-            // index of v[0] in the (m, q) tile: bit i of the lane selected the upper half at step i
+            // index of v[0] in the (m, q) tile after the scatter: bit i of the lane selects the upper
+            // half at step i
             int base = 0;
             {
                 int n = NV;
@@ -393,6 +393,14 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             // lanes that differ only in the bits above the halving steps hold the same sums; the one
             // whose high bits are zero stores them
             const bool owner = (lane >> kSteps) == 0;
+            // bias values are requested before the lane tree so that their latency hides behind it
+            float bv[kKeep];
+#pragma unroll
+            for (int t = 0; t < kKeep; ++t) {
+                const int n = un.tile * C::kRB + wr * RT + (base + t) % RT;
+                bv[t] = (direct && bias != nullptr && owner && n < N) ? __ldg(bias + n) : 0.0f;
+            }
+            lane_tree_scatter<MT * RT>(v, lane);
             // the output buffer may still be read by the previous kernel in the stream
             if (!waited) { pdl_wait(); waited = true; }
             if (owner) {
@@ -404,7 +412,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                     if (m < M && n < N) {
                         float r0 = v[t];
                         if (direct) {
-                            if (bias) r0 = __fadd_rn(r0, bias[n]);
+                            if (bias) r0 = __fadd_rn(r0, bv[t]);
                             out[(long long)m * N + n] = r0;
                         } else {
                             out[((long long)un.s * M + m) * N + n] = r0;
