@@ -120,7 +120,8 @@ DET_API det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream
 /* Copy the plan's order parameters to *out. */
 DET_API det_status_t det_linear_plan_get_params(const det_linear_plan_t* plan, det_linear_params_t* out);
 
-/* Write a JSON description (bucket, V, L, P, S, seg_len, order_version, kernel, workspace_bytes)
+/* Write a JSON description (bucket, V, L, P, S, seg_len, order_version, kernel, workspace_bytes and,
+ * for the decode kernel, the tiling the scheduler would pick on the current device -- schedule only)
  * to buf (at most n bytes including the terminator).  DET_ERR_INVALID_ARG if it does not fit. */
 DET_API det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, size_t n);
 

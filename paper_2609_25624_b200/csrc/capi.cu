@@ -213,11 +213,19 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
     if (!plan || !buf || n == 0) { set_error("describe: NULL argument"); return DET_ERR_INVALID_ARG; }
     const det_linear_params_t& p = plan->prm;
     static const char* kn[] = {"generic", "decode", "prefill"};
+    char tiling[96] = "null";
+    if (p.kernel == kKernelDecode) {
+        DecodeConfig c;
+        if (decode_config_for(p.M, p.N, p.K, plan->variant, &c))
+            snprintf(tiling, sizeof tiling, "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"kc\": %d, \"stages\": %d}", c.mt,
+                     c.wm, c.rt, c.wr, c.kc, c.stages);
+    }
     int w = snprintf(buf, n,
                      "{\"M\": %lld, \"N\": %lld, \"K\": %lld, \"bucket\": \"%s\", \"V\": %d, \"L\": %d, \"P\": %d, "
-                     "\"seg_len\": %lld, \"S\": %d, \"order_version\": %d, \"kernel\": \"%s\", \"workspace_bytes\": %llu}",
+                     "\"seg_len\": %lld, \"S\": %d, \"order_version\": %d, \"kernel\": \"%s\", \"workspace_bytes\": %llu, "
+                     "\"decode_tiling\": %s}",
                      (long long)p.M, (long long)p.N, (long long)p.K, p.bucket == 0 ? "decode" : "prefill", p.V, p.L, p.P,
-                     (long long)p.seg_len, p.S, p.order_version, kn[p.kernel], (unsigned long long)p.workspace_bytes);
+                     (long long)p.seg_len, p.S, p.order_version, kn[p.kernel], (unsigned long long)p.workspace_bytes, tiling);
     if (w < 0 || (size_t)w >= n) { set_error("describe: buffer too small (%d bytes needed)", w + 1); return DET_ERR_INVALID_ARG; }
     return DET_OK;
 }

@@ -202,13 +202,15 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 struct Unit {
     int tile, s, mb, k_lo, k_hi;
 };
-__device__ __forceinline__ Unit decode_unit(long long u, int n_row_tiles, int S, int seg_len, int K)
+// Work unit u -> (batch block fastest, then row tile, then segment): the batch blocks of one row tile
+// run side by side, so the tile's weights come from HBM once and from L2 for the other blocks.
+__device__ __forceinline__ Unit decode_unit(long long u, int n_row_tiles, int n_mblocks, int seg_len, int K)
 {
     Unit r;
-    r.tile = (int)(u % n_row_tiles);
-    const long long q = u / n_row_tiles;
-    r.s = (int)(q % S);
-    r.mb = (int)(q / S);
+    r.mb = (int)(u % n_mblocks);
+    const long long q = u / n_mblocks;
+    r.tile = (int)(q % n_row_tiles);
+    r.s = (int)(q / n_row_tiles);
     r.k_lo = r.s * seg_len;
     r.k_hi = min(K, r.k_lo + seg_len);
     return r;
@@ -263,7 +265,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                 long long u = blockIdx.x;
                 unsigned j = 0;
                 while (u < total_units && j < (unsigned)STAGES) {
-                    const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
+                    const Unit un = decode_unit(u, n_row_tiles, n_mblocks, seg_len, K);
                     for (int k0 = un.k_lo; k0 < un.k_hi && j < (unsigned)STAGES; k0 += KC, ++j) {
                         const uint32_t fb = full0 + 8 * j;
                         mbar_arrive_expect_tx(fb, C::kStageBytes);
@@ -278,7 +280,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             }
             pdl_wait();
             for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
-                const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
+                const Unit un = decode_unit(u, n_row_tiles, n_mblocks, seg_len, K);
                 const int n0 = un.tile * C::kRB;
                 for (int k0 = un.k_lo; k0 < un.k_hi; k0 += KC, ++it) {
                     const int st = it % STAGES;
@@ -315,7 +317,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         bool ok = true;
         bool waited = false;
         for (long long u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
-            const Unit un = decode_unit(u, n_row_tiles, S, seg_len, K);
+            const Unit un = decode_unit(u, n_row_tiles, n_mblocks, seg_len, K);
 
             float2 acc[MT][RT / 2];      // [m][j] = chains of outputs (m, row 2j) and (m, row 2j+1)
 #pragma unroll

@@ -29,14 +29,27 @@ double tiling_cost(const DecodeEntry& e, int64_t M, int64_t N, int S, int sm_cou
     const int64_t rb = (int64_t)c.rt * c.wr, mb = (int64_t)c.mt * c.wm;
     const int64_t units = ((N + rb - 1) / rb) * S * ((M + mb - 1) / mb);
     const int64_t per_sm = (units + sm_count - 1) / sm_count;
-    const double rows = (double)per_sm * (double)rb;
+    const double outputs = (double)per_sm * (double)rb * (double)mb;      // padded outputs on the busiest SM
     const int64_t resident = per_sm < occ ? per_sm : occ;
     const double warps = (double)resident * c.wm * c.wr;
     const double latency_penalty = warps >= 8.0 ? 1.0 : 8.0 / warps;
     // shared-memory wavefronts per packed FMA of an (mt x rt) warp tile
     const double r = (4.0 * c.mt + 2.0 * c.rt) / ((double)c.mt * c.rt);
     const double weight = M >= 8 ? 0.35 : 0.35 * (double)M / 8.0;
-    return rows * latency_penalty * (1.0 + weight * r);
+    // walking the batch in several blocks re-reads the weights from L2 and repeats the epilogue
+    const double block_penalty = 1.0 + 0.12 * (double)((M + mb - 1) / mb - 1);
+    return outputs * latency_penalty * block_penalty * (1.0 + weight * r);
+}
+
+// Tilings that can serve batch size M: those of M's own class and, for M > 8, the 8-row tilings
+// (the batch is then walked in blocks of 8 rows that run side by side).
+int candidate_classes(int64_t M, int* out)
+{
+    const int cls = m_class(M);
+    int n = 0;
+    out[n++] = cls;
+    if (cls > 3) out[n++] = 3;
+    return n;
 }
 
 }  // namespace
@@ -48,13 +61,16 @@ int decode_num_variants()
     return n;
 }
 
+// variant 0 = automatic; variant v >= 1 = the v-th candidate tiling for this batch size (own class
+// first, then the 8-row tilings when M > 8).
 bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfig* out)
 {
-    (void)K;
-    const int cls = m_class(M);
-    const DecodeClassTable* t = class_table(cls);
-    if (variant < 0 || variant > t->count) return false;
-    int pick = variant - 1;
+    int classes[2];
+    const int n_classes = candidate_classes(M, classes);
+    int total = 0;
+    for (int i = 0; i < n_classes; ++i) total += class_table(classes[i])->count;
+    if (variant < 0 || variant > total) return false;
+    int pick_cls = classes[0], pick = 0;
     if (variant == 0) {
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -64,14 +80,23 @@ bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfi
         det_linear_params_t prm;
         const int S = fill_params(M, N, K, &prm) == DET_OK ? prm.S : 1;
         double best = 1e301;
-        pick = 0;
-        for (int i = 0; i < t->count; ++i) {
-            const double c = tiling_cost(t->entries[i], M, N, S, sms);
-            if (c < best) { best = c; pick = i; }
+        for (int ci = 0; ci < n_classes; ++ci) {
+            const DecodeClassTable* t = class_table(classes[ci]);
+            for (int i = 0; i < t->count; ++i) {
+                const double c = tiling_cost(t->entries[i], M, N, S, sms);
+                if (c < best) { best = c; pick_cls = classes[ci]; pick = i; }
+            }
+        }
+    } else {
+        int v = variant - 1;
+        for (int ci = 0; ci < n_classes; ++ci) {
+            const DecodeClassTable* t = class_table(classes[ci]);
+            if (v < t->count) { pick_cls = classes[ci]; pick = v; break; }
+            v -= t->count;
         }
     }
-    *out = t->entries[pick].cfg;
-    out->id = cls * 64 + pick;
+    *out = class_table(pick_cls)->entries[pick].cfg;
+    out->id = pick_cls * 64 + pick;
     return true;
 }
 
