@@ -110,6 +110,14 @@ DET_API det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x
                                  const float* b, float* y_host, void* stream);
 
 /*
+ * The same without the final wait: the copies and kernels are only enqueued; y_host is valid once
+ * the caller has synchronised `stream`.  x_host must stay unchanged and y_host untouched until then;
+ * pinned host memory is needed for the copies to be asynchronous.  One call in flight per plan.
+ */
+DET_API det_status_t det_linear_run_host_async(det_linear_plan_t* plan, const float* x_host, const uint16_t* W,
+                                       const float* b, float* y_host, void* stream);
+
+/*
  * Synchronise `stream` and report whether any kernel launched through this plan gave up a bounded
  * device-side wait (every wait on a TMA completion barrier is limited; on expiry the kernel
  * records the fact and returns instead of spinning).  DET_OK, DET_ERR_DEVICE_TIMEOUT or

@@ -56,6 +56,8 @@ def lib() -> ctypes.CDLL:
         L.det_linear_run.restype = i32
         L.det_linear_run_host.argtypes = [p, p, p, p, p, p]
         L.det_linear_run_host.restype = i32
+        L.det_linear_run_host_async.argtypes = [p, p, p, p, p, p]
+        L.det_linear_run_host_async.restype = i32
         L.det_linear_plan_check.argtypes = [p, p]
         L.det_linear_plan_check.restype = i32
         L.det_linear_plan_get_params.argtypes = [p, ctypes.POINTER(Params)]
@@ -177,17 +179,22 @@ def det_linear_run(plan: Plan, x, W, b, y, stream=None) -> None:
                                 y.data_ptr(), _stream_ptr(stream)))
 
 
-def det_linear_run_host(plan: Plan, x_host, W, b, y_host, stream=None) -> None:
-    """x_host / y_host are (pinned) CPU tensors; W, b are CUDA tensors.  Synchronises the stream."""
+def det_linear_run_host(plan: Plan, x_host, W, b, y_host, stream=None, sync: bool = True) -> None:
+    """x_host / y_host are (pinned) CPU tensors; W, b are CUDA tensors.  Synchronises the stream
+    unless sync=False (then it calls det_linear_run_host_async and the caller synchronises)."""
     for t, shape, name in ((x_host, (plan.M, plan.K), "x_host"), (y_host, (plan.M, plan.N), "y_host")):
         if t.is_cuda or t.dtype != torch.float32 or tuple(t.shape) != shape or not t.is_contiguous():
             raise ValueError(f"{name}: need a contiguous CPU float32 tensor of shape {shape}")
     _expect(W, torch.bfloat16, (plan.N, plan.K), "W")
     if b is not None:
         _expect(b, torch.float32, (plan.N,), "b")
-    _check(lib().det_linear_run_host(plan.handle, x_host.data_ptr(), W.data_ptr(),
-                                     b.data_ptr() if b is not None else None, y_host.data_ptr(),
-                                     _stream_ptr(stream)))
+    fn = lib().det_linear_run_host if sync else lib().det_linear_run_host_async
+    _check(fn(plan.handle, x_host.data_ptr(), W.data_ptr(), b.data_ptr() if b is not None else None,
+              y_host.data_ptr(), _stream_ptr(stream)))
+
+
+def det_linear_run_host_async(plan: Plan, x_host, W, b, y_host, stream=None) -> None:
+    det_linear_run_host(plan, x_host, W, b, y_host, stream=stream, sync=False)
 
 
 def det_linear_run_noalloc(x, W, b, y, stream=None) -> None:

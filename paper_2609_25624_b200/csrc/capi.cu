@@ -62,6 +62,11 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const ui
                                cudaStream_t stream)
 {
     const det_linear_params_t& p = plan->prm;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != plan->device) {
+        set_error("run: the plan belongs to device %d but device %d is current", plan->device, dev);
+        return DET_ERR_INVALID_ARG;
+    }
     LaunchArgs a{};
     a.x = x; a.W = W; a.b = b; a.y = y;
     a.partials = plan->partials;
@@ -74,7 +79,7 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const ui
     a.variant = plan->variant;
 
     int kernel = plan->forced_kernel >= 0 ? plan->forced_kernel : p.kernel;
-    const bool fast_ok = (p.K % 8 == 0) && aligned16(x) && aligned16(W) && aligned16(y);
+    const bool fast_ok = (p.K % 8 == 0) && p.K <= (1 << 30) && p.N <= (1 << 30) && aligned16(x) && aligned16(W) && aligned16(y);
     if (!fast_ok) kernel = kKernelGeneric;
 
     cudaError_t e = cudaSuccess;
@@ -158,8 +163,8 @@ det_status_t det_linear_run(const det_linear_plan_t* plan, const float* x, const
     return run_device(const_cast<det_linear_plan_t*>(plan), x, W, b, y, static_cast<cudaStream_t>(stream));
 }
 
-det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, const uint16_t* W, const float* b,
-                                 float* y_host, void* stream)
+static det_status_t run_host_impl(det_linear_plan_t* plan, const float* x_host, const uint16_t* W, const float* b,
+                                  float* y_host, void* stream, bool sync)
 {
     if (!plan || !x_host || !W || !y_host) {
         set_error("run_host: plan, x_host, W and y_host must not be NULL");
@@ -180,9 +185,23 @@ det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, c
     if (s != DET_OK) return s;
     e = cudaMemcpyAsync(y_host, plan->y_stage, yb, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail("run_host: copy of y", e);
-    e = cudaStreamSynchronize(st);
-    if (e != cudaSuccess) return cuda_fail("run_host: synchronise", e);
+    if (sync) {
+        e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail("run_host: synchronise", e);
+    }
     return DET_OK;
+}
+
+det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, const uint16_t* W, const float* b,
+                                 float* y_host, void* stream)
+{
+    return run_host_impl(plan, x_host, W, b, y_host, stream, true);
+}
+
+det_status_t det_linear_run_host_async(det_linear_plan_t* plan, const float* x_host, const uint16_t* W, const float* b,
+                                       float* y_host, void* stream)
+{
+    return run_host_impl(plan, x_host, W, b, y_host, stream, false);
 }
 
 det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream)

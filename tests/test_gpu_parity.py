@@ -163,6 +163,10 @@ def test_run_host_matches_device_run():
     yh = torch.empty(M, N, dtype=torch.float32).pin_memory()
     B.det_linear_run_host(plan, xh, W.cuda(), b.cuda(), yh)
     assert_bits_equal(yh.numpy(), want, "run_host")
+    yh.zero_()
+    B.det_linear_run_host_async(plan, xh, W.cuda(), b.cuda(), yh)
+    torch.cuda.current_stream().synchronize()
+    assert_bits_equal(yh.numpy(), want, "run_host_async")
     plan.close()
 
 
