@@ -331,28 +331,40 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                 const uint32_t xs = smem_base + st * C::kStageBytes + (wm * MT) * (KC * 4) + lane * 16;
                 const uint32_t ws = smem_base + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * 8;
                 // One 128-element chunk: the lane's four elements of every row / batch row of the warp tile.
+                // Row pairs are processed in passes of at most four pairs so that only a few widened
+                // weights are live at a time (the accumulators already take most of the registers).
                 auto chunk = [&](int cc) {
-                    uint2 w[RT];
                     float4 xv[MT];
 #pragma unroll
-                    for (int q = 0; q < RT; ++q) w[q] = lds64(ws + q * (KC * 2) + cc * 256);
-#pragma unroll
                     for (int m = 0; m < MT; ++m) xv[m] = lds128(xs + m * (KC * 4) + cc * 512);
+                    constexpr int kPairs = RT / 2;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {          // the lane's four elements, ascending
-                        float2 wp[RT / 2];
+                    for (int p0 = 0; p0 < kPairs; p0 += 4) {
+                        constexpr int kMaxPass = 4;
+                        const int np = (kPairs - p0) < kMaxPass ? (kPairs - p0) : kMaxPass;   // compile-time after unrolling
+                        uint2 w[2 * kMaxPass];
 #pragma unroll
-                        for (int j = 0; j < RT / 2; ++j) {
-                            const uint32_t wa = (kk < 2) ? w[2 * j].x : w[2 * j].y;
-                            const uint32_t wb = (kk < 2) ? w[2 * j + 1].x : w[2 * j + 1].y;
-                            wp[j] = (kk & 1) ? make_float2(up_hi(wa), up_hi(wb)) : make_float2(up_lo(wa), up_lo(wb));
-                        }
+                        for (int q = 0; q < 2 * kMaxPass; ++q)
+                            if (q < 2 * np) w[q] = lds64(ws + (2 * p0 + q) * (KC * 2) + cc * 256);
 #pragma unroll
-                        for (int m = 0; m < MT; ++m) {
-                            const float xk = kk == 0 ? xv[m].x : kk == 1 ? xv[m].y : kk == 2 ? xv[m].z : xv[m].w;
-                            const float2 x2 = make_float2(xk, xk);
+                        for (int kk = 0; kk < 4; ++kk) {          // the lane's four elements, ascending
+                            float2 wp[kMaxPass];
 #pragma unroll
-                            for (int j = 0; j < RT / 2; ++j) acc[m][j] = __ffma2_rn(x2, wp[j], acc[m][j]);
+                            for (int j = 0; j < kMaxPass; ++j) {
+                                if (j < np) {
+                                    const uint32_t wa = (kk < 2) ? w[2 * j].x : w[2 * j].y;
+                                    const uint32_t wb = (kk < 2) ? w[2 * j + 1].x : w[2 * j + 1].y;
+                                    wp[j] = (kk & 1) ? make_float2(up_hi(wa), up_hi(wb)) : make_float2(up_lo(wa), up_lo(wb));
+                                }
+                            }
+#pragma unroll
+                            for (int m = 0; m < MT; ++m) {
+                                const float xk = kk == 0 ? xv[m].x : kk == 1 ? xv[m].y : kk == 2 ? xv[m].z : xv[m].w;
+                                const float2 x2 = make_float2(xk, xk);
+#pragma unroll
+                                for (int j = 0; j < kMaxPass; ++j)
+                                    if (j < np) acc[m][p0 + j] = __ffma2_rn(x2, wp[j], acc[m][p0 + j]);
+                            }
                         }
                     }
                 };
