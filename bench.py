@@ -322,7 +322,7 @@ def run_own(args, world, rank, local):
     else:
         line["cpu_baseline"] = cpu_baseline(work)
     # DRAM traffic per launch: ncu (dram__bytes_read.sum + dram__bytes_write.sum) on N = K = 4096 captures gives
-    # 1.000 / 0.997 / 0.987 x the algorithmic bytes at M = 1 / 8 / 32 (profiles/decode_kernel_4096x4096_ncu.md);
+    # 1.000 / 0.997 / 0.987 x the algorithmic bytes at M = 1 / 8 / 32 (ncu summaries under profiles/);
     # traffic is proportional to the algorithmic bytes, so it is scaled to the step's average launch here.
     line["roofline"]["traffic"] = DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes / launches_per_step
     line["roofline"]["algorithmic_bytes_per_launch"] = alg_bytes / launches_per_step

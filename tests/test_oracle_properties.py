@@ -126,7 +126,7 @@ def test_order_params_rule():
         ref = oracle.order_params(1, N, K)
         for M in (2, 8, 31, 32, 33, 64):
             assert oracle.order_params(M, N, K) == ref
-    # BASELINE shapes
+    # benchmark shapes
     assert oracle.order_params(1, 1024, 512) == dict(bucket="decode", V=4, L=32, P=1, seg_len=256, S=2,
                                                      order_version=1)
     for (N, K) in [(4096, 4096), (6144, 4096), (28672, 4096), (4096, 14336), (128256, 4096)]:
