@@ -53,6 +53,46 @@ float det_oracle_up(uint16_t h)
     return f;
 }
 
+/* Weight formats (the paper's probes cover BF16 and FP32 weights; its abstract speaks of "16-bit
+ * weights", which also admits IEEE binary16).  Every format widens exactly to binary32. */
+enum { ORACLE_W_BF16 = 0, ORACLE_W_FP16 = 1, ORACLE_W_FP32 = 2 };
+
+/* up() for IEEE binary16: every binary16 value (subnormals included) is a binary32 value. */
+float det_oracle_up_fp16(uint16_t h)
+{
+    const uint32_t sign = ((uint32_t)h & 0x8000u) << 16;
+    const uint32_t e = (h >> 10) & 0x1Fu;
+    const uint32_t m = h & 0x3FFu;
+    uint32_t bits;
+    if (e == 0) {
+        if (m == 0) {
+            bits = sign;                                   /* signed zero */
+        } else {
+            /* subnormal: m * 2^-24, normalised by hand */
+            uint32_t mm = m;
+            int shift = 0;
+            while ((mm & 0x400u) == 0) { mm <<= 1; ++shift; }
+            bits = sign | ((uint32_t)(113 - shift) << 23) | ((mm & 0x3FFu) << 13);
+        }
+    } else if (e == 31) {
+        bits = sign | 0x7F800000u | (m << 13);            /* infinity / NaN */
+    } else {
+        bits = sign | ((e + 112u) << 23) | (m << 13);
+    }
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+static inline float oracle_weight(const void *wrow, int64_t k, int wfmt)
+{
+    if (wfmt == ORACLE_W_FP32) return ((const float *)wrow)[k];
+    if (wfmt == ORACLE_W_FP16) return det_oracle_up_fp16(((const uint16_t *)wrow)[k]);
+    return det_oracle_up(((const uint16_t *)wrow)[k]);
+}
+
+static inline size_t oracle_weight_bytes(int wfmt) { return wfmt == ORACLE_W_FP32 ? 4 : 2; }
+
 /* Gradual underflow must be on: flush-to-zero / denormals-are-zero would change results for
  * subnormal operands (R1 asks for IEEE-754 arithmetic).  Returns the previous control word. */
 static unsigned oracle_enter_ieee(void)
@@ -75,7 +115,7 @@ static void oracle_leave_ieee(unsigned old)
 }
 
 /* One output element y[m,n]: xrow = x[m,:], wrow = W[n,:], bias = &b[n] or NULL. */
-static float oracle_one(const float *xrow, const uint16_t *wrow, const float *bias,
+static float oracle_one(const float *xrow, const void *wrow, int wfmt, const float *bias,
                         int64_t K, int V, int L, int P, int64_t seg_len)
 {
     float a[ORACLE_MAX_LEAVES];
@@ -93,7 +133,7 @@ static float oracle_one(const float *xrow, const uint16_t *wrow, const float *bi
                     int64_t k = c + (int64_t)l * V + j;
                     if (k < k_hi) {
                         int leaf = l * P + (j % P);
-                        a[leaf] = fmaf(xrow[k], det_oracle_up(wrow[k]), a[leaf]);
+                        a[leaf] = fmaf(xrow[k], oracle_weight(wrow, k, wfmt), a[leaf]);
                     }
                 }
             }
@@ -115,13 +155,15 @@ static int oracle_args_ok(int64_t M, int64_t N, int64_t K, int V, int L, int P, 
     return 1;
 }
 
-/* Full problem.  x: [M,K] row-major FP32; W: [N,K] row-major BF16 bit patterns; b: [N] or NULL;
- * y: [M,N] row-major.  Returns 0 on success, 1 on bad arguments. */
-int det_oracle_linear(const float *x, const uint16_t *W, const float *b, float *y,
-                      int64_t M, int64_t N, int64_t K,
-                      int V, int L, int P, int64_t seg_len, int nthreads)
+/* Full problem.  x: [M,K] row-major FP32; W: [N,K] row-major in the given weight format (BF16 or
+ * FP16 bit patterns, or FP32 values); b: [N] or NULL; y: [M,N] row-major.  Returns 0 on success, 1 on
+ * bad arguments. */
+int det_oracle_linear_w(const float *x, const void *W, int wfmt, const float *b, float *y,
+                        int64_t M, int64_t N, int64_t K,
+                        int V, int L, int P, int64_t seg_len, int nthreads)
 {
-    if (!oracle_args_ok(M, N, K, V, L, P, seg_len)) return 1;
+    if (!oracle_args_ok(M, N, K, V, L, P, seg_len) || wfmt < 0 || wfmt > 2) return 1;
+    const size_t wb = oracle_weight_bytes(wfmt);
 #ifdef _OPENMP
     if (nthreads < 1) nthreads = omp_get_max_threads();
 #else
@@ -133,22 +175,31 @@ int det_oracle_linear(const float *x, const uint16_t *W, const float *b, float *
         #pragma omp for schedule(static)
         for (int64_t n = 0; n < N; ++n)
             for (int64_t m = 0; m < M; ++m)
-                y[m * N + n] = oracle_one(x + m * K, W + n * K, b ? b + n : NULL, K, V, L, P, seg_len);
+                y[m * N + n] = oracle_one(x + m * K, (const char *)W + (size_t)n * K * wb, wfmt, b ? b + n : NULL,
+                                          K, V, L, P, seg_len);
         oracle_leave_ieee(csr);
     }
     return 0;
 }
 
+int det_oracle_linear(const float *x, const uint16_t *W, const float *b, float *y,
+                      int64_t M, int64_t N, int64_t K,
+                      int V, int L, int P, int64_t seg_len, int nthreads)
+{
+    return det_oracle_linear_w(x, W, ORACLE_W_BF16, b, y, M, N, K, V, L, P, seg_len, nthreads);
+}
+
 /* Selected outputs only: out[i] = y[ms[i], ns[i]] (for full-size problems where the whole matrix
  * would take too long). */
-int det_oracle_linear_sampled(const float *x, const uint16_t *W, const float *b,
-                              const int64_t *ms, const int64_t *ns, int64_t count, float *out,
-                              int64_t M, int64_t N, int64_t K,
-                              int V, int L, int P, int64_t seg_len, int nthreads)
+int det_oracle_linear_sampled_w(const float *x, const void *W, int wfmt, const float *b,
+                                const int64_t *ms, const int64_t *ns, int64_t count, float *out,
+                                int64_t M, int64_t N, int64_t K,
+                                int V, int L, int P, int64_t seg_len, int nthreads)
 {
-    if (!oracle_args_ok(M, N, K, V, L, P, seg_len) || count < 0) return 1;
+    if (!oracle_args_ok(M, N, K, V, L, P, seg_len) || count < 0 || wfmt < 0 || wfmt > 2) return 1;
     for (int64_t i = 0; i < count; ++i)
         if (ms[i] < 0 || ms[i] >= M || ns[i] < 0 || ns[i] >= N) return 1;
+    const size_t wb = oracle_weight_bytes(wfmt);
 #ifdef _OPENMP
     if (nthreads < 1) nthreads = omp_get_max_threads();
 #else
@@ -159,10 +210,19 @@ int det_oracle_linear_sampled(const float *x, const uint16_t *W, const float *b,
         unsigned csr = oracle_enter_ieee();
         #pragma omp for schedule(static)
         for (int64_t i = 0; i < count; ++i)
-            out[i] = oracle_one(x + ms[i] * K, W + ns[i] * K, b ? b + ns[i] : NULL, K, V, L, P, seg_len);
+            out[i] = oracle_one(x + ms[i] * K, (const char *)W + (size_t)ns[i] * K * wb, wfmt, b ? b + ns[i] : NULL,
+                                K, V, L, P, seg_len);
         oracle_leave_ieee(csr);
     }
     return 0;
+}
+
+int det_oracle_linear_sampled(const float *x, const uint16_t *W, const float *b,
+                              const int64_t *ms, const int64_t *ns, int64_t count, float *out,
+                              int64_t M, int64_t N, int64_t K,
+                              int V, int L, int P, int64_t seg_len, int nthreads)
+{
+    return det_oracle_linear_sampled_w(x, W, ORACLE_W_BF16, b, ms, ns, count, out, M, N, K, V, L, P, seg_len, nthreads);
 }
 
 /* Greedy argmax per row with the lower index winning a tie (the tie rule stated in the end-to-end

@@ -22,6 +22,11 @@ def bf16_bits_to_float(h: int) -> float:
     return struct.unpack("<f", struct.pack("<I", (h & 0xFFFF) << 16))[0]
 
 
+def fp16_bits_to_float(h: int) -> float:
+    """up() for IEEE binary16 bit patterns (exact: every binary16 value is a binary32 value)."""
+    return struct.unpack("<e", struct.pack("<H", h & 0xFFFF))[0]
+
+
 def round_to_binary32(q: Fraction) -> float:
     """Round an exact rational to the nearest binary32, ties to even, gradual underflow,
     overflow to infinity (IEEE-754 roundTiesToEven)."""
@@ -78,13 +83,14 @@ def add32(a: float, b: float) -> float:
     return round_to_binary32(q)
 
 
-def output(xrow, wrow, bias, V, L, P, seg_len):
-    """One output element.  xrow: binary32-representable floats; wrow: BF16 bit patterns (ints);
-    bias: float or None.  Follows the order family (V, L, P, seg_len): chunks of V*L elements
+def output(xrow, wrow, bias, V, L, P, seg_len, wfmt="bf16"):
+    """One output element.  xrow: binary32-representable floats; wrow: BF16 or FP16 bit patterns
+    (ints) or, for wfmt="fp32", binary32-representable floats; bias: float or None.  Follows the order family (V, L, P, seg_len): chunks of V*L elements
     ascending, lane l owns V consecutive elements, element j feeds sub-chain j mod P, leaves are
     tree-summed adjacent-first, segments are summed ascending, bias is added last."""
     K = len(xrow)
     assert len(wrow) == K
+    decode = {"bf16": bf16_bits_to_float, "fp16": fp16_bits_to_float, "fp32": float}[wfmt]
     nleaf = L * P
     assert nleaf & (nleaf - 1) == 0
     C = V * L
@@ -100,7 +106,7 @@ def output(xrow, wrow, bias, V, L, P, seg_len):
                     k = c + l * V + j
                     if k < k_hi:
                         leaf = l * P + (j % P)
-                        a[leaf] = fma32(xrow[k], bf16_bits_to_float(wrow[k]), a[leaf])
+                        a[leaf] = fma32(xrow[k], decode(wrow[k]), a[leaf])
             c += C
         w = nleaf
         while w > 1:
@@ -111,8 +117,9 @@ def output(xrow, wrow, bias, V, L, P, seg_len):
     return add32(t, bias) if bias is not None else t
 
 
-def linear(x, W_bits, b, V, L, P, seg_len):
+def linear(x, W_bits, b, V, L, P, seg_len, wfmt="bf16"):
     """Whole (tiny) problem as nested lists: y[m][n]."""
-    return [[output(list(map(float, xr)), list(map(int, wr)), None if b is None else float(b[n]),
-                    V, L, P, seg_len)
+    conv = float if wfmt == "fp32" else int
+    return [[output(list(map(float, xr)), list(map(conv, wr)), None if b is None else float(b[n]),
+                    V, L, P, seg_len, wfmt)
              for n, wr in enumerate(W_bits)] for xr in x]

@@ -90,6 +90,13 @@ def lib() -> ctypes.CDLL:
         L.det_oracle_linear_sampled.argtypes = [p, p, p, p, p, i64, p, i64, i64, i64,
                                                 i32, i32, i32, i64, i32]
         L.det_oracle_linear_sampled.restype = i32
+        L.det_oracle_linear_w.argtypes = [p, p, i32, p, p, i64, i64, i64, i32, i32, i32, i64, i32]
+        L.det_oracle_linear_w.restype = i32
+        L.det_oracle_linear_sampled_w.argtypes = [p, p, i32, p, p, p, i64, p, i64, i64, i64,
+                                                  i32, i32, i32, i64, i32]
+        L.det_oracle_linear_sampled_w.restype = i32
+        L.det_oracle_up_fp16.argtypes = [ctypes.c_uint16]
+        L.det_oracle_up_fp16.restype = ctypes.c_float
         L.det_oracle_argmax_rows.argtypes = [p, i64, i64, p]
         L.det_oracle_argmax_rows.restype = i32
         L.det_oracle_up.argtypes = [ctypes.c_uint16]
@@ -105,9 +112,16 @@ def _f32(a, shape):
     return a
 
 
-def _bf16_bits(W, shape):
+#: weight formats: 16-bit formats are passed as bit patterns (uint16), FP32 weights as float32
+WEIGHT_FORMATS = {"bf16": 0, "fp16": 1, "fp32": 2}
+
+
+def _weights(W, shape, wfmt):
     W = np.ascontiguousarray(W)
-    assert W.dtype == np.uint16, "W must be given as BF16 bit patterns (uint16)"
+    if wfmt == "fp32":
+        assert W.dtype == np.float32, "FP32 weights must be a float32 array"
+    else:
+        assert W.dtype == np.uint16, "16-bit weights must be given as bit patterns (uint16)"
     assert W.shape == shape, (W.shape, shape)
     return W
 
@@ -117,33 +131,33 @@ def _resolve(M, N, K, params):
     return int(prm["V"]), int(prm["L"]), int(prm["P"]), int(prm["seg_len"])
 
 
-def linear(x, W_bits, b=None, params=None, threads=0):
-    """y = x . up(W)^T (+ b) in the frozen order.  x [M,K] float32, W_bits [N,K] uint16 (BF16 bit
-    patterns), b [N] float32 or None.  `params` overrides the shape-derived order (for the scaled-
-    down hand examples)."""
+def linear(x, W_bits, b=None, params=None, threads=0, wfmt="bf16"):
+    """y = x . up(W)^T (+ b) in the frozen order.  x [M,K] float32, W_bits [N,K] uint16 (BF16 or FP16
+    bit patterns) or float32 (wfmt="fp32"), b [N] float32 or None.  `params` overrides the
+    shape-derived order (for the scaled-down hand examples)."""
     x = np.ascontiguousarray(x, dtype=np.float32)
     M, K = x.shape
     N = W_bits.shape[0]
-    W_bits = _bf16_bits(W_bits, (N, K))
+    W_bits = _weights(W_bits, (N, K), wfmt)
     V, L, P, seg_len = _resolve(M, N, K, params)
     y = np.empty((M, N), dtype=np.float32)
     bp = None
     if b is not None:
         b = _f32(b, (N,))
         bp = b.ctypes.data
-    rc = lib().det_oracle_linear(x.ctypes.data, W_bits.ctypes.data, bp, y.ctypes.data,
-                                 M, N, K, V, L, P, seg_len, threads)
+    rc = lib().det_oracle_linear_w(x.ctypes.data, W_bits.ctypes.data, WEIGHT_FORMATS[wfmt], bp, y.ctypes.data,
+                                   M, N, K, V, L, P, seg_len, threads)
     if rc != 0:
-        raise ValueError("det_oracle_linear rejected its arguments")
+        raise ValueError("det_oracle_linear_w rejected its arguments")
     return y
 
 
-def linear_sampled(x, W_bits, b, ms, ns, params=None, threads=0):
+def linear_sampled(x, W_bits, b, ms, ns, params=None, threads=0, wfmt="bf16"):
     """Selected outputs y[ms[i], ns[i]] of the same computation."""
     x = np.ascontiguousarray(x, dtype=np.float32)
     M, K = x.shape
     N = W_bits.shape[0]
-    W_bits = _bf16_bits(W_bits, (N, K))
+    W_bits = _weights(W_bits, (N, K), wfmt)
     V, L, P, seg_len = _resolve(M, N, K, params)
     ms = np.ascontiguousarray(ms, dtype=np.int64)
     ns = np.ascontiguousarray(ns, dtype=np.int64)
@@ -152,11 +166,11 @@ def linear_sampled(x, W_bits, b, ms, ns, params=None, threads=0):
     if b is not None:
         b = _f32(b, (N,))
         bp = b.ctypes.data
-    rc = lib().det_oracle_linear_sampled(x.ctypes.data, W_bits.ctypes.data, bp, ms.ctypes.data,
-                                         ns.ctypes.data, ms.shape[0], out.ctypes.data,
-                                         M, N, K, V, L, P, seg_len, threads)
+    rc = lib().det_oracle_linear_sampled_w(x.ctypes.data, W_bits.ctypes.data, WEIGHT_FORMATS[wfmt], bp,
+                                           ms.ctypes.data, ns.ctypes.data, ms.shape[0], out.ctypes.data,
+                                           M, N, K, V, L, P, seg_len, threads)
     if rc != 0:
-        raise ValueError("det_oracle_linear_sampled rejected its arguments")
+        raise ValueError("det_oracle_linear_sampled_w rejected its arguments")
     return out
 
 
@@ -173,6 +187,10 @@ def argmax_rows(y):
 
 def up(h: int) -> float:
     return float(lib().det_oracle_up(int(h) & 0xFFFF))
+
+
+def up_fp16(h: int) -> float:
+    return float(lib().det_oracle_up_fp16(int(h) & 0xFFFF))
 
 
 def threads() -> int:

@@ -159,3 +159,57 @@ def test_tail_elements_are_skipped_not_zero_filled():
     W1 = np.array([[0x0001]], dtype=np.uint16)
     y1 = oracle.linear(x1, W1, None, params=dict(V=4, L=1, P=1, seg_len=256))   # 3 skipped elements
     assert y1.view(np.uint32)[0, 0] == 0x80000000
+
+
+def test_up_fp16_all_bit_patterns():
+    """Binary16 -> binary32 widening of the oracle: all 65 536 patterns against numpy's own
+    float16 -> float32 conversion (NaNs compared as NaNs)."""
+    hs = np.arange(65536, dtype=np.uint16)
+    want = hs.view(np.float16).astype(np.float32)
+    got = np.array([oracle.up_fp16(int(h)) for h in hs], dtype=np.float32)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan].view(np.uint32), want[~nan].view(np.uint32))
+    for h in (0x0001, 0x03FF, 0x0400, 0x7BFF, 0x8001, 0xFBFF, 0x3C00):
+        assert exact.fp16_bits_to_float(h) == oracle.up_fp16(h)
+
+
+@pytest.mark.parametrize("wfmt", ["fp16", "fp32"])
+def test_other_weight_formats_follow_the_same_order(wfmt):
+    """FP16 and FP32 weights go through the same reduction order: hand-traced examples with all
+    weights = 1 give the same values, the C oracle equals the exact micro-oracle on random tiny
+    cases, and values exactly representable in BF16 give bit-identical results in every format."""
+    one = {"fp16": 0x3C00, "fp32": 1.0}[wfmt]
+    for e in EXAMPLES:
+        if any(w != gu.ONE_BF16 for w in e["w"]):
+            continue
+        K = len(e["x"])
+        seg = gu.seg_len_for(K, e["s_req"], e["granule"])
+        x = np.array([e["x"]], dtype=np.float32)
+        W = np.full((1, K), one, dtype=np.float32 if wfmt == "fp32" else np.uint16)
+        b = None if e["b"] is None else np.array([e["b"]], dtype=np.float32)
+        y = oracle.linear(x, W, b, params=dict(V=e["V"], L=e["L"], P=e["P"], seg_len=seg), wfmt=wfmt)
+        assert float(y[0, 0]) == e["expected"], e["name"]
+    rng = random.Random(77)
+    for case in range(25):
+        V, L, P = rng.choice([(1, 1, 1), (4, 32, 1), (2, 2, 2), (8, 32, 1)])
+        K = rng.choice([3, 8, 31, 100, 257])
+        seg = gu.seg_len_for(K, rng.choice([1, 2, 3]), max(V * L, 8) // (V * L) * (V * L) if V * L <= 8 else V * L)
+        x = [[_rand_f32(rng) for _ in range(K)] for _ in range(2)]
+        if wfmt == "fp16":
+            W = [[rng.choice([0x3C00, 0xBC00, 0x0000, 0x8000, 0x0001, 0x83FF, rng.randrange(0x2000, 0x5000),
+                              0x8000 | rng.randrange(0x2000, 0x5000)]) for _ in range(K)] for _ in range(3)]
+            Wa = np.array(W, dtype=np.uint16)
+        else:
+            W = [[_rand_f32(rng) for _ in range(K)] for _ in range(3)]
+            Wa = np.array(W, dtype=np.float32)
+        want = np.array(exact.linear(x, W, None, V, L, P, seg, wfmt), dtype=np.float32)
+        got = oracle.linear(np.array(x, dtype=np.float32), Wa, None, params=dict(V=V, L=L, P=P, seg_len=seg), wfmt=wfmt)
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), (case, V, L, P, K)
+    # BF16-exact values: identical bits whatever the storage format
+    g = np.random.default_rng(5)
+    Wb = (g.standard_normal((7, 640)).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    Wf = (Wb.astype(np.uint32) << 16).view(np.float32)
+    x = g.standard_normal((3, 640)).astype(np.float32)
+    ref = oracle.linear(x, Wb, None)
+    assert np.array_equal(oracle.linear(x, Wf, None, wfmt="fp32").view(np.uint32), ref.view(np.uint32))
