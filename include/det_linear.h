@@ -55,6 +55,15 @@ typedef enum {
     DET_ERR_ARCH = 7                /* current device is not sm_100                               */
 } det_status_t;
 
+/* Storage format of the weight matrix.  Every format widens exactly to FP32 in registers (Eq. 2's
+ * up()); the reduction order does not depend on it.  The paper's kernels take "16-bit weights" and
+ * its seeded probe covers BF16 and FP32 weights. */
+typedef enum {
+    DET_WEIGHT_BF16 = 0,            /* bfloat16 bit patterns, 2 bytes per element (default)        */
+    DET_WEIGHT_FP16 = 1,            /* IEEE binary16 bit patterns, 2 bytes per element             */
+    DET_WEIGHT_FP32 = 2             /* IEEE binary32, 4 bytes per element (no widening needed)     */
+} det_weight_format_t;
+
 /* Order parameters of a shape; filled by det_linear_plan_params / det_linear_plan_get_params. */
 typedef struct {
     int64_t M, N, K;
@@ -64,7 +73,7 @@ typedef struct {
     int32_t S;               /* number of segments, = ceil(K / seg_len)                             */
     int32_t order_version;   /* version of the order definition, 1                                  */
     int32_t kernel;          /* 0 generic, 1 decode (TMA pipeline), 2 prefill tile kernel           */
-    int32_t reserved;
+    int32_t weight_format;   /* det_weight_format_t of the plan (0 = BF16 for det_linear_plan_params)    */
     uint64_t workspace_bytes;/* split-K partials: 4*S*M*N bytes when S > 1, else 0                  */
 } det_linear_params_t;
 
@@ -84,6 +93,10 @@ DET_API det_status_t det_linear_plan_params(int64_t M, int64_t N, int64_t K, det
  */
 DET_API det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K);
 
+/* The same for a weight matrix stored as FP16 or FP32 (wfmt: det_weight_format_t).  The order
+ * parameters are those of det_linear_plan_params: they depend on the shape only. */
+DET_API det_linear_plan_t* det_linear_plan_w(int64_t M, int64_t N, int64_t K, int32_t wfmt);
+
 /*
  * Enqueue the computation on `stream` (a cudaStream_t; NULL = the legacy default stream) and
  * return without synchronising.  Eq. 2 with the order above; split-K partials, if any, are
@@ -100,13 +113,20 @@ DET_API det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K);
 DET_API det_status_t det_linear_run(const det_linear_plan_t* plan, const float* x, const uint16_t* W,
                             const float* b, float* y, void* stream);
 
+/* det_linear_run for any weight format: W points to [N,K] row-major elements of the plan's format
+ * (det_linear_run itself accepts BF16 and FP16 plans; an FP32 plan needs this entry point).  The fast
+ * kernels need 16-byte aligned buffers and a 16-byte row pitch (K % 8 == 0 for 16-bit weights,
+ * K % 4 == 0 for FP32 weights). */
+DET_API det_status_t det_linear_run_w(const det_linear_plan_t* plan, const float* x, const void* W,
+                              const float* b, float* y, void* stream);
+
 /*
  * End-to-end variant with HOST activations: copies x (host, [M,K]) to a plan-owned device buffer,
- * runs the same kernels, copies y back to y_host (host, [M,N]) and waits for the stream.  W and b
- * stay device-resident (they are the model's parameters).  The staging buffers are allocated on
+ * runs the same kernels, copies y back to y_host (host, [M,N]) and waits for the stream.  W (in the
+ * plan's weight format) and b stay device-resident (they are the model's parameters).  The staging buffers are allocated on
  * first use.  Synchronises `stream` before returning.
  */
-DET_API det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, const uint16_t* W,
+DET_API det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, const void* W,
                                  const float* b, float* y_host, void* stream);
 
 /*
@@ -114,7 +134,7 @@ DET_API det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x
  * the caller has synchronised `stream`.  x_host must stay unchanged and y_host untouched until then;
  * pinned host memory is needed for the copies to be asynchronous.  One call in flight per plan.
  */
-DET_API det_status_t det_linear_run_host_async(det_linear_plan_t* plan, const float* x_host, const uint16_t* W,
+DET_API det_status_t det_linear_run_host_async(det_linear_plan_t* plan, const float* x_host, const void* W,
                                        const float* b, float* y_host, void* stream);
 
 /*

@@ -30,7 +30,7 @@ class Params(ctypes.Structure):
     _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
                 ("bucket", ctypes.c_int32), ("V", ctypes.c_int32), ("L", ctypes.c_int32), ("P", ctypes.c_int32),
                 ("seg_len", ctypes.c_int64), ("S", ctypes.c_int32), ("order_version", ctypes.c_int32),
-                ("kernel", ctypes.c_int32), ("reserved", ctypes.c_int32), ("workspace_bytes", ctypes.c_uint64)]
+                ("kernel", ctypes.c_int32), ("weight_format", ctypes.c_int32), ("workspace_bytes", ctypes.c_uint64)]
 
     def as_dict(self):
         return {"bucket": "decode" if self.bucket == 0 else "prefill", "V": self.V, "L": self.L, "P": self.P,
@@ -52,8 +52,12 @@ def lib() -> ctypes.CDLL:
         L.det_linear_plan_params.restype = i32
         L.det_linear_plan.argtypes = [i64, i64, i64]
         L.det_linear_plan.restype = p
+        L.det_linear_plan_w.argtypes = [i64, i64, i64, ctypes.c_int32]
+        L.det_linear_plan_w.restype = p
         L.det_linear_run.argtypes = [p, p, p, p, p, p]
         L.det_linear_run.restype = i32
+        L.det_linear_run_w.argtypes = [p, p, p, p, p, p]
+        L.det_linear_run_w.restype = i32
         L.det_linear_run_host.argtypes = [p, p, p, p, p, p]
         L.det_linear_run_host.restype = i32
         L.det_linear_run_host_async.argtypes = [p, p, p, p, p, p]
@@ -117,12 +121,23 @@ def _stream_ptr(stream):
     return stream.cuda_stream
 
 
+# det_weight_format_t and the torch dtype that carries each format
+DET_WEIGHT_BF16, DET_WEIGHT_FP16, DET_WEIGHT_FP32 = 0, 1, 2
+WEIGHT_DTYPES = {DET_WEIGHT_BF16: torch.bfloat16, DET_WEIGHT_FP16: torch.float16, DET_WEIGHT_FP32: torch.float32}
+WEIGHT_FORMATS = {"bf16": DET_WEIGHT_BF16, "fp16": DET_WEIGHT_FP16, "fp32": DET_WEIGHT_FP32}
+
+
 class Plan:
     """Owner of a det_linear_plan_t*."""
 
-    def __init__(self, M: int, N: int, K: int):
+    def __init__(self, M: int, N: int, K: int, wfmt: int = DET_WEIGHT_BF16):
         self.M, self.N, self.K = int(M), int(N), int(K)
-        self._h = lib().det_linear_plan(self.M, self.N, self.K)
+        self.wfmt = WEIGHT_FORMATS.get(wfmt, wfmt) if isinstance(wfmt, str) else int(wfmt)
+        self.w_dtype = WEIGHT_DTYPES.get(self.wfmt, torch.bfloat16)
+        if self.wfmt == DET_WEIGHT_BF16:
+            self._h = lib().det_linear_plan(self.M, self.N, self.K)
+        else:
+            self._h = lib().det_linear_plan_w(self.M, self.N, self.K, self.wfmt)
         if not self._h:
             raise DetLinearError(-1, det_last_error())
 
@@ -144,6 +159,11 @@ class Plan:
 
 def det_linear_plan(M: int, N: int, K: int) -> Plan:
     return Plan(M, N, K)
+
+
+def det_linear_plan_w(M: int, N: int, K: int, wfmt) -> Plan:
+    """Plan for weights stored as "bf16" / "fp16" / "fp32" (or the det_weight_format_t value)."""
+    return Plan(M, N, K, wfmt)
 
 
 def det_linear_plan_destroy(plan: Plan) -> None:
@@ -171,12 +191,24 @@ def _expect(t, dtype, shape, name):
 def det_linear_run(plan: Plan, x, W, b, y, stream=None) -> None:
     """Enqueue y = x . up(W)^T (+ b) on `stream` (default: torch's current stream)."""
     _expect(x, torch.float32, (plan.M, plan.K), "x")
-    _expect(W, torch.bfloat16, (plan.N, plan.K), "W")
+    _expect(W, plan.w_dtype, (plan.N, plan.K), "W")
     _expect(y, torch.float32, (plan.M, plan.N), "y")
     if b is not None:
         _expect(b, torch.float32, (plan.N,), "b")
-    _check(lib().det_linear_run(plan.handle, x.data_ptr(), W.data_ptr(), b.data_ptr() if b is not None else None,
-                                y.data_ptr(), _stream_ptr(stream)))
+    fn = lib().det_linear_run if plan.wfmt == DET_WEIGHT_BF16 else lib().det_linear_run_w
+    _check(fn(plan.handle, x.data_ptr(), W.data_ptr(), b.data_ptr() if b is not None else None,
+              y.data_ptr(), _stream_ptr(stream)))
+
+
+def det_linear_run_w(plan: Plan, x, W, b, y, stream=None) -> None:
+    """det_linear_run for a plan of any weight format (always through the det_linear_run_w entry)."""
+    _expect(x, torch.float32, (plan.M, plan.K), "x")
+    _expect(W, plan.w_dtype, (plan.N, plan.K), "W")
+    _expect(y, torch.float32, (plan.M, plan.N), "y")
+    if b is not None:
+        _expect(b, torch.float32, (plan.N,), "b")
+    _check(lib().det_linear_run_w(plan.handle, x.data_ptr(), W.data_ptr(), b.data_ptr() if b is not None else None,
+                                  y.data_ptr(), _stream_ptr(stream)))
 
 
 def det_linear_run_host(plan: Plan, x_host, W, b, y_host, stream=None, sync: bool = True) -> None:
@@ -185,7 +217,7 @@ def det_linear_run_host(plan: Plan, x_host, W, b, y_host, stream=None, sync: boo
     for t, shape, name in ((x_host, (plan.M, plan.K), "x_host"), (y_host, (plan.M, plan.N), "y_host")):
         if t.is_cuda or t.dtype != torch.float32 or tuple(t.shape) != shape or not t.is_contiguous():
             raise ValueError(f"{name}: need a contiguous CPU float32 tensor of shape {shape}")
-    _expect(W, torch.bfloat16, (plan.N, plan.K), "W")
+    _expect(W, plan.w_dtype, (plan.N, plan.K), "W")
     if b is not None:
         _expect(b, torch.float32, (plan.N,), "b")
     fn = lib().det_linear_run_host if sync else lib().det_linear_run_host_async

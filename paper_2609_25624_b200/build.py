@@ -14,8 +14,10 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libdet_linear.so")
 OBJ_DIR = os.path.join(HERE, "csrc", "obj")
 
-SOURCES = ["plan.cpp", "capi.cu", "kernels_generic.cu", "kernels_decode.cu", "decode_inst_0.cu", "decode_inst_1.cu", "decode_inst_2.cu",
-           "decode_inst_3.cu", "kernels_prefill.cu", "bench_kernels.cu", "noalloc.cu"]
+# (source, extra defines): the decode tilings are compiled once per weight format
+SOURCES = [("plan.cpp", ()), ("capi.cu", ()), ("kernels_generic.cu", ()), ("kernels_decode.cu", ()),
+           ("kernels_prefill.cu", ()), ("bench_kernels.cu", ()), ("noalloc.cu", ())]
+SOURCES += [(f"decode_inst_{i}.cu", (f"-DDET_WF={wf}",)) for wf in (0, 1, 2) for i in range(4)]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -38,12 +40,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers += [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE) if f.endswith(".h")]
     objs, procs = [], []
-    for src in SOURCES:
+    for src, defines in SOURCES:
         sp = os.path.join(CSRC, src)
-        op = os.path.join(OBJ_DIR, os.path.splitext(src)[0] + ".o")
+        tag = "".join(d.replace("-D", "_").replace("=", "") for d in defines)
+        op = os.path.join(OBJ_DIR, os.path.splitext(src)[0] + tag + ".o")
         objs.append(op)
         if force or _stale(op, [sp] + headers):
-            cmd = [nvcc, *NVCC_FLAGS, "-x", "cu", "-c", sp, "-o", op]
+            cmd = [nvcc, *NVCC_FLAGS, *defines, "-x", "cu", "-c", sp, "-o", op]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))

@@ -58,7 +58,7 @@ static bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, 
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-static det_status_t run_device(det_linear_plan_t* plan, const float* x, const uint16_t* W, const float* b, float* y,
+static det_status_t run_device(det_linear_plan_t* plan, const float* x, const void* W, const float* b, float* y,
                                cudaStream_t stream)
 {
     const det_linear_params_t& p = plan->prm;
@@ -69,6 +69,7 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const ui
     }
     LaunchArgs a{};
     a.x = x; a.W = W; a.b = b; a.y = y;
+    a.wfmt = p.weight_format;
     a.partials = plan->partials;
     a.M = p.M; a.N = p.N; a.K = p.K;
     a.seg_len = p.seg_len; a.S = p.S;
@@ -79,24 +80,28 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const ui
     a.variant = plan->variant;
 
     int kernel = plan->forced_kernel >= 0 ? plan->forced_kernel : p.kernel;
-    const bool fast_ok = (p.K % 8 == 0) && p.K <= (1 << 30) && p.N <= (1 << 30) && aligned16(x) && aligned16(W) && aligned16(y);
+    const int64_t k_align = p.weight_format == DET_WEIGHT_FP32 ? 4 : 8;     // 16-byte row pitch of W (x: K % 4)
+    const bool fast_ok = (p.K % k_align == 0) && (p.K % 4 == 0) && p.K <= (1 << 30) && p.N <= (1 << 30) && aligned16(x) && aligned16(W) && aligned16(y);
     if (!fast_ok) kernel = kKernelGeneric;
 
     cudaError_t e = cudaSuccess;
     if (kernel == kKernelDecode) {
         DecodeConfig cfg;
-        if (!decode_config_for(p.M, p.N, p.K, plan->variant, &cfg)) {
+        if (!decode_config_for(p.M, p.N, p.K, p.weight_format, plan->variant, &cfg)) {
             set_error("run: no decode configuration for this shape/variant");
             return DET_ERR_INVALID_ARG;
         }
-        if (plan->map_w_ptr != W || plan->map_x_ptr != x || plan->map_cfg_id != cfg.id) {
-            if (!encode_2d(&plan->map_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)p.N, (uint64_t)p.K,
+        if (plan->map_w_ptr != W || plan->map_x_ptr != x || plan->map_cfg_id != cfg.id + 1024 * p.weight_format) {
+            const CUtensorMapDataType wdt = p.weight_format == DET_WEIGHT_FP32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                            : p.weight_format == DET_WEIGHT_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                                                 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+            if (!encode_2d(&plan->map_w, wdt, p.weight_format == DET_WEIGHT_FP32 ? 4 : 2, W, (uint64_t)p.N, (uint64_t)p.K,
                            (uint32_t)cfg.rt, (uint32_t)cfg.kc, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
                 return DET_ERR_CUDA;
             if (!encode_2d(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, x, (uint64_t)p.M, (uint64_t)p.K,
                            (uint32_t)(cfg.mt * cfg.wm), (uint32_t)cfg.kc, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
                 return DET_ERR_CUDA;
-            plan->map_w_ptr = W; plan->map_x_ptr = x; plan->map_cfg_id = cfg.id;
+            plan->map_w_ptr = W; plan->map_x_ptr = x; plan->map_cfg_id = cfg.id + 1024 * p.weight_format;
         }
         e = launch_decode(a, &plan->map_w, &plan->map_x);
     } else if (kernel == kKernelPrefill) {
@@ -119,10 +124,15 @@ det_status_t det_linear_plan_params(int64_t M, int64_t N, int64_t K, det_linear_
     return fill_params(M, N, K, out);
 }
 
-det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K)
+det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K) { return det_linear_plan_w(M, N, K, DET_WEIGHT_BF16); }
+
+det_linear_plan_t* det_linear_plan_w(int64_t M, int64_t N, int64_t K, int32_t wfmt)
 {
     det_linear_params_t prm;
     if (fill_params(M, N, K, &prm) != DET_OK) return nullptr;
+    if (wfmt < DET_WEIGHT_BF16 || wfmt > DET_WEIGHT_FP32) { set_error("plan: unknown weight format %d", wfmt); return nullptr; }
+    prm.weight_format = wfmt;
+    if (wfmt == DET_WEIGHT_FP32) prm.kernel = (K % 4 == 0) ? (prm.bucket == 0 ? kKernelDecode : kKernelPrefill) : kKernelGeneric;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) { cuda_fail("cudaGetDevice", e); return nullptr; }
@@ -158,12 +168,22 @@ det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K)
 det_status_t det_linear_run(const det_linear_plan_t* plan, const float* x, const uint16_t* W, const float* b, float* y,
                             void* stream)
 {
+    if (plan && plan->prm.weight_format == DET_WEIGHT_FP32) {
+        set_error("run: the plan stores FP32 weights; use det_linear_run_w");
+        return DET_ERR_INVALID_ARG;
+    }
+    return det_linear_run_w(plan, x, W, b, y, stream);
+}
+
+det_status_t det_linear_run_w(const det_linear_plan_t* plan, const float* x, const void* W, const float* b, float* y,
+                              void* stream)
+{
     if (!plan || !x || !W || !y) { set_error("run: plan, x, W and y must not be NULL"); return DET_ERR_INVALID_ARG; }
     // the plan's tensor-map cache is the only state a run touches
     return run_device(const_cast<det_linear_plan_t*>(plan), x, W, b, y, static_cast<cudaStream_t>(stream));
 }
 
-static det_status_t run_host_impl(det_linear_plan_t* plan, const float* x_host, const uint16_t* W, const float* b,
+static det_status_t run_host_impl(det_linear_plan_t* plan, const float* x_host, const void* W, const float* b,
                                   float* y_host, void* stream, bool sync)
 {
     if (!plan || !x_host || !W || !y_host) {
@@ -192,13 +212,13 @@ static det_status_t run_host_impl(det_linear_plan_t* plan, const float* x_host, 
     return DET_OK;
 }
 
-det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, const uint16_t* W, const float* b,
+det_status_t det_linear_run_host(det_linear_plan_t* plan, const float* x_host, const void* W, const float* b,
                                  float* y_host, void* stream)
 {
     return run_host_impl(plan, x_host, W, b, y_host, stream, true);
 }
 
-det_status_t det_linear_run_host_async(det_linear_plan_t* plan, const float* x_host, const uint16_t* W, const float* b,
+det_status_t det_linear_run_host_async(det_linear_plan_t* plan, const float* x_host, const void* W, const float* b,
                                        float* y_host, void* stream)
 {
     return run_host_impl(plan, x_host, W, b, y_host, stream, false);
@@ -232,19 +252,20 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
     if (!plan || !buf || n == 0) { set_error("describe: NULL argument"); return DET_ERR_INVALID_ARG; }
     const det_linear_params_t& p = plan->prm;
     static const char* kn[] = {"generic", "decode", "prefill"};
-    char tiling[96] = "null";
+    char tiling[128] = "null";
     if (p.kernel == kKernelDecode) {
         DecodeConfig c;
-        if (decode_config_for(p.M, p.N, p.K, plan->variant, &c))
+        if (decode_config_for(p.M, p.N, p.K, p.weight_format, plan->variant, &c))
             snprintf(tiling, sizeof tiling, "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"kc\": %d, \"stages\": %d}", c.mt,
                      c.wm, c.rt, c.wr, c.kc, c.stages);
     }
     int w = snprintf(buf, n,
                      "{\"M\": %lld, \"N\": %lld, \"K\": %lld, \"bucket\": \"%s\", \"V\": %d, \"L\": %d, \"P\": %d, "
                      "\"seg_len\": %lld, \"S\": %d, \"order_version\": %d, \"kernel\": \"%s\", \"workspace_bytes\": %llu, "
-                     "\"decode_tiling\": %s}",
+                     "\"weight_format\": \"%s\", \"decode_tiling\": %s}",
                      (long long)p.M, (long long)p.N, (long long)p.K, p.bucket == 0 ? "decode" : "prefill", p.V, p.L, p.P,
-                     (long long)p.seg_len, p.S, p.order_version, kn[p.kernel], (unsigned long long)p.workspace_bytes, tiling);
+                     (long long)p.seg_len, p.S, p.order_version, kn[p.kernel], (unsigned long long)p.workspace_bytes,
+                     p.weight_format == DET_WEIGHT_FP32 ? "fp32" : p.weight_format == DET_WEIGHT_FP16 ? "fp16" : "bf16", tiling);
     if (w < 0 || (size_t)w >= n) { set_error("describe: buffer too small (%d bytes needed)", w + 1); return DET_ERR_INVALID_ARG; }
     return DET_OK;
 }
@@ -299,7 +320,7 @@ det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
     if (!plan || variant < 0) { set_error("set_variant: bad argument"); return DET_ERR_INVALID_ARG; }
     if (plan->prm.bucket == 0) {
         DecodeConfig cfg;
-        if (!decode_config_for(plan->prm.M, plan->prm.N, plan->prm.K, variant, &cfg)) {
+        if (!decode_config_for(plan->prm.M, plan->prm.N, plan->prm.K, plan->prm.weight_format, variant, &cfg)) {
             set_error("set_variant: the decode kernel has fewer than %d tilings for this batch size", variant);
             return DET_ERR_INVALID_ARG;
         }

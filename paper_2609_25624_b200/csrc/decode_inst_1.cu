@@ -1,9 +1,24 @@
-// Tilings of the decode kernel for one or more batch classes (all numerically identical).
+// Tilings of the decode kernel for one or more batch classes (all numerically identical).  Compiled once
+// per weight format (DET_WF = 0 BF16, 1 FP16, 2 FP32); FP32 weights take twice the shared memory per
+// stage, so their lists use narrower stages.
 #include "decode_kernel.cuh"
 
 namespace detlin {
 using namespace decode_detail;
 
+#define DET_TABLE_NAME2(cls, wf) DET_TABLE_NAME(cls, wf)
+
+#if DET_WF == 2
+static const DecodeEntry kEntries3[] = {
+    DEC(8, 1, 4, 4, 128, 5, 1),
+    DEC(8, 1, 6, 4, 128, 4, 1),
+    DEC(8, 1, 8, 4, 128, 4, 1),
+    DEC(8, 1, 10, 4, 128, 3, 1),
+    DEC(8, 1, 12, 4, 128, 3, 4),
+    DEC(8, 1, 14, 4, 128, 3, 4),
+    DEC(8, 1, 8, 2, 128, 6, 1),
+};
+#else
 static const DecodeEntry kEntries3[] = {
     DEC(8, 1, 4, 4, 256, 5, 1),
     DEC(8, 1, 6, 4, 256, 4, 1),
@@ -14,6 +29,7 @@ static const DecodeEntry kEntries3[] = {
     DEC(8, 1, 16, 4, 256, 3, 4),
     DEC(8, 1, 8, 2, 256, 6, 1),
 };
-const DecodeClassTable kDecodeClass3 = {kEntries3, 8};
+#endif
+extern const DecodeClassTable DET_TABLE_NAME2(3, DET_WF) = {kEntries3, (int)(sizeof(kEntries3) / sizeof(kEntries3[0]))};
 
 }  // namespace detlin

@@ -110,16 +110,38 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// The four consecutive weights of one row that a lane owns in a chunk: one 8-byte load for the
+// 16-bit formats, one 16-byte load for FP32; element kk widened exactly to FP32.
+template <int WF> struct WVec { typedef uint2 type; };
+template <> struct WVec<2> { typedef float4 type; };
+template <int WF>
+__device__ __forceinline__ typename WVec<WF>::type wload(uint32_t addr)
+{
+    if constexpr (WF == 2) return lds128(addr);
+    else return lds64(addr);
+}
+template <int WF>
+__device__ __forceinline__ float wget(const typename WVec<WF>::type& v, int kk)
+{
+    if constexpr (WF == 2) {
+        return kk == 0 ? v.x : kk == 1 ? v.y : kk == 2 ? v.z : v.w;
+    } else {
+        const uint32_t w = (kk < 2) ? v.x : v.y;
+        return (kk & 1) ? up16_hi<WF>(w) : up16_lo<WF>(w);
+    }
+}
+
 // PG = warps in the producer group: 1 (plain) or 4 (a whole warpgroup, which lets the kernel move
 // registers from the producer to the consumers with setmaxnreg when the consumer tile is large).
-template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
+template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG, int WF>
 struct Cfg {
     static constexpr int kConsumerWarps = WM * WR;
     static constexpr int kThreads = (kConsumerWarps + PG) * 32;
     static constexpr int kMB = MT * WM;                       // batch rows per x box
     static constexpr int kRB = RT * WR;                       // weight rows per block tile
     static constexpr int kXBytes = kMB * KC * 4;
-    static constexpr int kWBoxBytes = RT * KC * 2;
+    static constexpr int kEB = WeightElem<WF>::bytes;         // bytes per weight element
+    static constexpr int kWBoxBytes = RT * KC * kEB;
     static constexpr int kStageBytes = kXBytes + WR * kWBoxBytes;
     static constexpr int kBarBytes = 256;                     // 2*STAGES barriers + abort flag
     static constexpr int kSmemBytes = STAGES * kStageBytes + kBarBytes + 128;   // +128 for alignment
@@ -137,6 +159,7 @@ struct Cfg {
     static_assert(PG == 1 || kConsumerRegs * kConsumerWarps * 32 + kProducerRegs * PG * 32 <= kThreads * kLaunchRegs,
                   "register move must fit in the block's own allocation");
     static_assert(PG == 1 || kConsumerRegs >= kLaunchRegs, "consumers only ever grow");
+    static_assert(kSmemBytes <= 227 * 1024, "a block's ring must fit in shared memory");
     static_assert(RT % 2 == 0, "weight rows are processed in pairs (one FP32x2 accumulator per pair)");
     static_assert(PG == 1 || (PG == 4 && kConsumerWarps % 4 == 0), "setmaxnreg works on whole warpgroups");
     static_assert(STAGES >= 2 && STAGES <= 12, "ring depth");
@@ -216,13 +239,13 @@ __device__ __forceinline__ Unit decode_unit(long long u, int n_row_tiles, int n_
     return r;
 }
 
-template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
-__global__ void __launch_bounds__((WM * WR + PG) * 32, (Cfg<MT, WM, RT, WR, KC, STAGES, PG>::kMinBlocks))
+template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG, int WF>
+__global__ void __launch_bounds__((WM * WR + PG) * 32, (Cfg<MT, WM, RT, WR, KC, STAGES, PG, WF>::kMinBlocks))
 decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
               const float* __restrict__ bias, float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct,
               int n_row_tiles, int n_mblocks, DeviceStatus* status)
 {
-    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG>;
+    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG, WF>;
     extern __shared__ unsigned char smem_raw[];
     // 128-byte aligned base (TMA destination requirement)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -329,7 +352,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                 const int st = it % STAGES;
                 if (!mbar_wait(full0 + 8 * st, (it / STAGES) & 1, abort_flag, status, 2)) { ok = false; break; }
                 const uint32_t xs = smem_base + st * C::kStageBytes + (wm * MT) * (KC * 4) + lane * 16;
-                const uint32_t ws = smem_base + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * 8;
+                const uint32_t ws = smem_base + st * C::kStageBytes + C::kXBytes + wr * C::kWBoxBytes + lane * (4 * C::kEB);
                 // One 128-element chunk: the lane's four elements of every row / batch row of the warp tile.
                 // Row pairs are processed in passes of at most four pairs so that only a few widened
                 // weights are live at a time (the accumulators already take most of the registers).
@@ -342,20 +365,16 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                     for (int p0 = 0; p0 < kPairs; p0 += 4) {
                         constexpr int kMaxPass = 4;
                         const int np = (kPairs - p0) < kMaxPass ? (kPairs - p0) : kMaxPass;   // compile-time after unrolling
-                        uint2 w[2 * kMaxPass];
+                        typename WVec<WF>::type w[2 * kMaxPass];
 #pragma unroll
                         for (int q = 0; q < 2 * kMaxPass; ++q)
-                            if (q < 2 * np) w[q] = lds64(ws + (2 * p0 + q) * (KC * 2) + cc * 256);
+                            if (q < 2 * np) w[q] = wload<WF>(ws + (2 * p0 + q) * (KC * C::kEB) + cc * (128 * C::kEB));
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk) {          // the lane's four elements, ascending
                             float2 wp[kMaxPass];
 #pragma unroll
                             for (int j = 0; j < kMaxPass; ++j) {
-                                if (j < np) {
-                                    const uint32_t wa = (kk < 2) ? w[2 * j].x : w[2 * j].y;
-                                    const uint32_t wb = (kk < 2) ? w[2 * j + 1].x : w[2 * j + 1].y;
-                                    wp[j] = (kk & 1) ? make_float2(up_hi(wa), up_hi(wb)) : make_float2(up_lo(wa), up_lo(wb));
-                                }
+                                if (j < np) wp[j] = make_float2(wget<WF>(w[2 * j], kk), wget<WF>(w[2 * j + 1], kk));
                             }
 #pragma unroll
                             for (int m = 0; m < MT; ++m) {
@@ -444,13 +463,13 @@ typedef int (*DecodeOccupancyFn)();
 
 // Resident blocks per SM of one tiling (also opts the kernel into its dynamic shared memory).
 // Returns 0 if the query fails.
-template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
+template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG, int WF>
 int decode_occupancy_t()
 {
-    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG>;
+    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG, WF>;
     static int blocks_per_sm = -1;
     if (blocks_per_sm < 0) {
-        auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES, PG>;
+        auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES, PG, WF>;
         int occ = 0;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess ||
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, C::kThreads, C::kSmemBytes) != cudaSuccess) {
@@ -462,12 +481,12 @@ int decode_occupancy_t()
     return blocks_per_sm;
 }
 
-template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG>
+template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG, int WF>
 cudaError_t launch_decode_t(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
 {
-    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG>;
-    auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES, PG>;
-    const int blocks_per_sm = decode_occupancy_t<MT, WM, RT, WR, KC, STAGES, PG>();
+    using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG, WF>;
+    auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES, PG, WF>;
+    const int blocks_per_sm = decode_occupancy_t<MT, WM, RT, WR, KC, STAGES, PG, WF>();
     if (blocks_per_sm <= 0) return cudaErrorLaunchOutOfResources;
     const int n_row_tiles = (int)((a.N + C::kRB - 1) / C::kRB);
     const int n_mblocks = (int)((a.M + C::kMB - 1) / C::kMB);
@@ -500,17 +519,28 @@ struct DecodeEntry {
     DecodeOccupancyFn occupancy;
 };
 
+#ifndef DET_WF
+#define DET_WF 0
+#endif
 #define DEC(MT, WM, RT, WR, KC, ST, PG) \
-    { {MT, WM, RT, WR, KC, ST, 0}, &launch_decode_t<MT, WM, RT, WR, KC, ST, PG>, &decode_occupancy_t<MT, WM, RT, WR, KC, ST, PG> }
+    { {MT, WM, RT, WR, KC, ST, 0}, &launch_decode_t<MT, WM, RT, WR, KC, ST, PG, DET_WF>, &decode_occupancy_t<MT, WM, RT, WR, KC, ST, PG, DET_WF> }
 
 }  // namespace decode_detail
 
-// One table of tilings per batch class, defined in the decode_inst_*.cu files (separate files only
-// to compile in parallel).  All entries of a class produce identical bits.
+// One table of tilings per weight format and batch class, defined in the decode_inst_*.cu files
+// (separate files, compiled once per format, only to build in parallel).  All entries of a class
+// produce identical bits.
 struct DecodeClassTable {
     const decode_detail::DecodeEntry* entries;
     int count;
 };
-extern const DecodeClassTable kDecodeClass0, kDecodeClass1, kDecodeClass2, kDecodeClass3, kDecodeClass4, kDecodeClass5;
+#define DET_CAT3(a, b, c) a##b##c
+#define DET_TABLE_NAME(cls, wf) DET_CAT3(kDecodeClass, cls, _wf##wf)
+#define DET_DECLARE_TABLES(wf)                                                                         \
+    extern const DecodeClassTable DET_TABLE_NAME(0, wf), DET_TABLE_NAME(1, wf), DET_TABLE_NAME(2, wf), \
+        DET_TABLE_NAME(3, wf), DET_TABLE_NAME(4, wf), DET_TABLE_NAME(5, wf);
+DET_DECLARE_TABLES(0)
+DET_DECLARE_TABLES(1)
+DET_DECLARE_TABLES(2)
 
 }  // namespace detlin

@@ -2,6 +2,7 @@
 // R1: never rely on the compiler's contraction), packed FP32x2 FMA, and the adjacent-first lane tree.
 #pragma once
 #include <cuda_runtime.h>
+#include <cuda_fp16.h>
 #include <cstdint>
 
 namespace detlin {
@@ -11,6 +12,30 @@ __device__ __forceinline__ float up_bf16(uint16_t h) { return __uint_as_float(((
 // A 32-bit word holding two BF16 values (little endian: element k in the low half, k+1 in the high).
 __device__ __forceinline__ float up_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float up_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Weight formats: WF = 0 BF16, 1 FP16, 2 FP32 (det_weight_format_t).  A 32-bit word of a 16-bit
+// format holds elements (k, k+1) in its (low, high) half; both widenings are exact.
+template <int WF>
+__device__ __forceinline__ float up16_lo(uint32_t w)
+{
+    if (WF == 0) return __uint_as_float(w << 16);
+    return __half2float(__ushort_as_half((unsigned short)(w & 0xffffu)));
+}
+template <int WF>
+__device__ __forceinline__ float up16_hi(uint32_t w)
+{
+    if (WF == 0) return __uint_as_float(w & 0xffff0000u);
+    return __half2float(__ushort_as_half((unsigned short)(w >> 16)));
+}
+template <int WF> struct WeightElem { typedef uint16_t type; static constexpr int bytes = 2; };
+template <> struct WeightElem<2> { typedef float type; static constexpr int bytes = 4; };
+template <int WF>
+__device__ __forceinline__ float up_elem(typename WeightElem<WF>::type v)
+{
+    if constexpr (WF == 2) return v;
+    else if constexpr (WF == 1) return __half2float(__ushort_as_half(v));
+    else return __uint_as_float(((uint32_t)v) << 16);
+}
 
 // fma.rn.f32x2: two independent IEEE-754 binary32 fused multiply-adds (round to nearest even, no
 // flush to zero) in one instruction; each half behaves exactly like fma.rn.f32.

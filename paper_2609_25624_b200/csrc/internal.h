@@ -26,7 +26,8 @@ det_status_t fill_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* o
 // ---- kernel launchers (defined in the .cu files) -------------------------------------------
 struct LaunchArgs {
     const float* x;
-    const uint16_t* W;
+    const void* W;        // [N,K] in weight format wfmt
+    int wfmt;             // det_weight_format_t
     const float* b;
     float* y;             // final output [M,N]
     float* partials;      // [S,M,N] when S > 1, else nullptr
@@ -53,7 +54,7 @@ struct DecodeConfig {
     int mt, wm, rt, wr, kc, stages;   // warp tile (mt x rt), warps (wm x wr), k per stage, ring depth
     int id;
 };
-bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfig* out);
+bool decode_config_for(int64_t M, int64_t N, int64_t K, int wfmt, int variant, DecodeConfig* out);
 int decode_num_variants();
 
 }  // namespace detlin

@@ -9,11 +9,14 @@ namespace {
 
 using decode_detail::DecodeEntry;
 
-const DecodeClassTable* class_table(int cls)
+#define DET_TABLE_ROW(wf)                                                                                  \
+    { &DET_TABLE_NAME(0, wf), &DET_TABLE_NAME(1, wf), &DET_TABLE_NAME(2, wf), &DET_TABLE_NAME(3, wf), \
+      &DET_TABLE_NAME(4, wf), &DET_TABLE_NAME(5, wf) }
+
+const DecodeClassTable* class_table(int wfmt, int cls)
 {
-    static const DecodeClassTable* const t[6] = {&kDecodeClass0, &kDecodeClass1, &kDecodeClass2,
-                                                 &kDecodeClass3, &kDecodeClass4, &kDecodeClass5};
-    return t[cls];
+    static const DecodeClassTable* const t[3][6] = {DET_TABLE_ROW(0), DET_TABLE_ROW(1), DET_TABLE_ROW(2)};
+    return t[wfmt][cls];
 }
 
 int m_class(int64_t M) { return M <= 1 ? 0 : M <= 2 ? 1 : M <= 4 ? 2 : M <= 8 ? 3 : M <= 16 ? 4 : 5; }
@@ -57,18 +60,18 @@ int candidate_classes(int64_t M, int* out)
 int decode_num_variants()
 {
     int n = 0;
-    for (int c = 0; c < 6; ++c) n = class_table(c)->count > n ? class_table(c)->count : n;
+    for (int c = 0; c < 6; ++c) n = class_table(0, c)->count > n ? class_table(0, c)->count : n;
     return n;
 }
 
 // variant 0 = automatic; variant v >= 1 = the v-th candidate tiling for this batch size (own class
 // first, then the 8-row tilings when M > 8).
-bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfig* out)
+bool decode_config_for(int64_t M, int64_t N, int64_t K, int wfmt, int variant, DecodeConfig* out)
 {
     int classes[2];
     const int n_classes = candidate_classes(M, classes);
     int total = 0;
-    for (int i = 0; i < n_classes; ++i) total += class_table(classes[i])->count;
+    for (int i = 0; i < n_classes; ++i) total += class_table(wfmt, classes[i])->count;
     if (variant < 0 || variant > total) return false;
     int pick_cls = classes[0], pick = 0;
     if (variant == 0) {
@@ -81,7 +84,7 @@ bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfi
         const int S = fill_params(M, N, K, &prm) == DET_OK ? prm.S : 1;
         double best = 1e301;
         for (int ci = 0; ci < n_classes; ++ci) {
-            const DecodeClassTable* t = class_table(classes[ci]);
+            const DecodeClassTable* t = class_table(wfmt, classes[ci]);
             for (int i = 0; i < t->count; ++i) {
                 const double c = tiling_cost(t->entries[i], M, N, S, sms);
                 if (c < best) { best = c; pick_cls = classes[ci]; pick = i; }
@@ -90,12 +93,12 @@ bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfi
     } else {
         int v = variant - 1;
         for (int ci = 0; ci < n_classes; ++ci) {
-            const DecodeClassTable* t = class_table(classes[ci]);
+            const DecodeClassTable* t = class_table(wfmt, classes[ci]);
             if (v < t->count) { pick_cls = classes[ci]; pick = v; break; }
             v -= t->count;
         }
     }
-    *out = class_table(pick_cls)->entries[pick].cfg;
+    *out = class_table(wfmt, pick_cls)->entries[pick].cfg;
     out->id = pick_cls * 64 + pick;
     return true;
 }
@@ -103,8 +106,8 @@ bool decode_config_for(int64_t M, int64_t N, int64_t K, int variant, DecodeConfi
 cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
 {
     DecodeConfig cfg;
-    if (!decode_config_for(a.M, a.N, a.K, a.variant, &cfg)) return cudaErrorInvalidValue;
-    return class_table(cfg.id / 64)->entries[cfg.id % 64].fn(a, map_w, map_x);
+    if (!decode_config_for(a.M, a.N, a.K, a.wfmt, a.variant, &cfg)) return cudaErrorInvalidValue;
+    return class_table(a.wfmt, cfg.id / 64)->entries[cfg.id % 64].fn(a, map_w, map_x);
 }
 
 }  // namespace detlin

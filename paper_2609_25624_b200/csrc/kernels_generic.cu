@@ -10,8 +10,9 @@ namespace detlin {
 // Decode order (V=4, L=32, P=1): one warp per (row n, segment s); lane l owns k = c + 4l + j in every
 // 128-element chunk and accumulates them in ascending order into one chain; the 32 lanes are summed
 // adjacent-first.
+template <int WF>
 __global__ void __launch_bounds__(256)
-generic_decode_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, const float* __restrict__ b,
+generic_decode_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type* __restrict__ W, const float* __restrict__ b,
                       float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct)
 {
     const int lane = threadIdx.x & 31;
@@ -21,7 +22,7 @@ generic_decode_kernel(const float* __restrict__ x, const uint16_t* __restrict__ 
     const int s = (int)(warp % S);
     const int64_t k_lo = (int64_t)s * seg_len;
     const int64_t k_hi = (k_lo + seg_len < K) ? k_lo + seg_len : K;
-    const uint16_t* wrow = W + n * K;
+    const typename WeightElem<WF>::type* wrow = W + n * K;
     for (int64_t m = 0; m < M; ++m) {
         const float* xrow = x + m * K;
         float a = 0.0f;
@@ -30,7 +31,7 @@ generic_decode_kernel(const float* __restrict__ x, const uint16_t* __restrict__ 
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int64_t k = k0 + j;
-                if (k < k_hi) a = __fmaf_rn(xrow[k], up_bf16(wrow[k]), a);
+                if (k < k_hi) a = __fmaf_rn(xrow[k], up_elem<WF>(wrow[k]), a);
             }
         }
         const float t = lane_tree_sum(a);
@@ -42,8 +43,9 @@ generic_decode_kernel(const float* __restrict__ x, const uint16_t* __restrict__ 
 }
 
 // Prefill order (V=1, L=1, P=1): one thread per (m, n, segment), one chain, strictly ascending k.
+template <int WF>
 __global__ void __launch_bounds__(256)
-generic_prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, const float* __restrict__ b,
+generic_prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type* __restrict__ W, const float* __restrict__ b,
                        float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct)
 {
     const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -53,9 +55,9 @@ generic_prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__
     const int64_t k_lo = (int64_t)s * seg_len;
     const int64_t k_hi = (k_lo + seg_len < K) ? k_lo + seg_len : K;
     const float* xrow = x + m * K;
-    const uint16_t* wrow = W + n * K;
+    const typename WeightElem<WF>::type* wrow = W + n * K;
     float t = 0.0f;
-    for (int64_t k = k_lo; k < k_hi; ++k) t = __fmaf_rn(xrow[k], up_bf16(wrow[k]), t);
+    for (int64_t k = k_lo; k < k_hi; ++k) t = __fmaf_rn(xrow[k], up_elem<WF>(wrow[k]), t);
     if (direct) out[m * N + n] = b ? __fadd_rn(t, b[n]) : t;
     else        out[((int64_t)s * M + m) * N + n] = t;
 }
@@ -73,15 +75,17 @@ combine_kernel(const float* __restrict__ partials, const float* __restrict__ b, 
     y[i] = b ? __fadd_rn(t, b[i % N]) : t;
 }
 
-cudaError_t launch_generic(const LaunchArgs& a, int bucket)
+template <int WF>
+static cudaError_t launch_generic_t(const LaunchArgs& a, int bucket)
 {
+    typedef typename WeightElem<WF>::type WT;
+    const WT* W = static_cast<const WT*>(a.W);
     const int direct = (a.S == 1);
     float* out = direct ? a.y : a.partials;
     if (bucket == 0) {
         const int64_t warps = a.N * a.S;
         const int64_t blocks = (warps + 7) / 8;
-        generic_decode_kernel<<<(unsigned)blocks, 256, 0, a.stream>>>(a.x, a.W, a.b, out, a.M, a.N, a.K,
-                                                                      a.seg_len, a.S, direct);
+        generic_decode_kernel<WF><<<(unsigned)blocks, 256, 0, a.stream>>>(a.x, W, a.b, out, a.M, a.N, a.K, a.seg_len, a.S, direct);
     } else {
         // grid.y carries M (< 65536 per launch); larger M is cut into slabs of rows
         const int64_t max_y = 32768;
@@ -89,14 +93,20 @@ cudaError_t launch_generic(const LaunchArgs& a, int bucket)
             const int64_t mm = (a.M - m0 < max_y) ? a.M - m0 : max_y;
             dim3 grid((unsigned)((a.N + 255) / 256), (unsigned)mm, (unsigned)a.S);
             float* o = out + m0 * a.N;   // both layouts ([M][N] and [s][M][N]) advance by whole rows
-            generic_prefill_kernel<<<grid, 256, 0, a.stream>>>(a.x + m0 * a.K, a.W, a.b, o, a.M, a.N, a.K,
-                                                              a.seg_len, a.S, direct);
+            generic_prefill_kernel<WF><<<grid, 256, 0, a.stream>>>(a.x + m0 * a.K, W, a.b, o, a.M, a.N, a.K, a.seg_len, a.S, direct);
         }
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (!direct) return launch_combine(a);
     return cudaSuccess;
+}
+
+cudaError_t launch_generic(const LaunchArgs& a, int bucket)
+{
+    if (a.wfmt == 1) return launch_generic_t<1>(a, bucket);
+    if (a.wfmt == 2) return launch_generic_t<2>(a, bucket);
+    return launch_generic_t<0>(a, bucket);
 }
 
 cudaError_t launch_combine(const LaunchArgs& a)

@@ -12,8 +12,8 @@
 // Schedule (numerically inert): 128 x 128 output tile per block, 256 threads, 8 x 8 outputs per
 // thread (4 column pairs), two blocks per SM, K walked in slabs of 32 with two slab buffers.  Both
 // operands are staged k-major ([k][m] and [k][n]) so that a thread reads its eight x values and its
-// eight weights of one k with four 16-byte loads.  BF16 weights are widened to FP32 once per block
-// while the slab is staged (HBM and L2 only ever carry BF16 weights, Eq. 2).  Global loads of slab
+// eight weights of one k with four 16-byte loads.  16-bit weights are widened to FP32 once per block
+// while the slab is staged (HBM and L2 only ever carry the stored format, Eq. 2).  Global loads of slab
 // i+1 are in flight while slab i is multiplied.
 #include "internal.h"
 #include "device_utils.cuh"
@@ -45,8 +45,10 @@ __device__ __forceinline__ uint4 ldg128_nc(const void* p)
     return v;
 }
 
+// WF: weight format (0 BF16, 1 FP16: octets of 16-bit weights; 2 FP32: quads, staged like x)
+template <int WF>
 __global__ void __launch_bounds__(kThreads, 2)
-prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, const float* __restrict__ bias,
+prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type* __restrict__ W, const float* __restrict__ bias,
                float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct, int tiles_m, int tiles_n)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -89,32 +91,36 @@ prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, cons
         xg[j] = x + (long long)(xok[j] ? m : 0) * K + q * 4;
         xs_off[j] = (uint32_t)((q * 4) * kPitch + r) * 4;
     }
-    const uint16_t* wg[2];
-    uint32_t ws_off[2];
-    int wk[2];
-    bool wok[2];
+    // FP32 weights: 128 rows x 8 quads, the same assignment as the x tile.
+    constexpr int NW = (WF == 2) ? 4 : 2;            // 16-byte pieces of W per thread and slab
+    constexpr int WE = (WF == 2) ? 4 : 8;            // weights per piece
+    const typename WeightElem<WF>::type* wg[NW];
+    uint32_t ws_off[NW];
+    int wk[NW];
+    bool wok[NW];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
+    for (int j = 0; j < NW; ++j) {
         const int p = tid + 256 * j;
         const int o = p & 1, r = (p >> 1) & 127, c = 2 * (p >> 8) + o;
         const int n = n0 + r;
         wok[j] = n < N;
-        wk[j] = c * 8;
-        wg[j] = W + (long long)(wok[j] ? n : 0) * K + c * 8;
-        ws_off[j] = (uint32_t)((c * 8) * kPitch + r) * 4;
+        wk[j] = c * WE;
+        wg[j] = W + (long long)(wok[j] ? n : 0) * K + c * WE;
+        ws_off[j] = (uint32_t)((c * WE) * kPitch + r) * 4;
     }
 
     uint4 xr[4];
-    uint4 wr[2];
+    uint4 wr[NW];
     auto load_slab = [&](int k0) {
-        // K % 8 == 0: an octet of weights / a quad of activations is entirely inside or outside [.., k_hi)
+        // the row pitch is a whole number of 16-byte pieces: a piece of weights / a quad of activations is
+        // entirely inside or outside [.., k_hi)
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             if (xok[j] && k0 + xk[j] < k_hi) xr[j] = ldg128_nc(xg[j] + k0);
             else xr[j] = make_uint4(0u, 0u, 0u, 0u);
         }
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < NW; ++j) {
             if (wok[j] && k0 + wk[j] < k_hi) wr[j] = ldg128_nc(wg[j] + k0);
             else wr[j] = make_uint4(0u, 0u, 0u, 0u);
         }
@@ -130,17 +136,24 @@ prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, cons
             sts32(a + 3 * kPitch * 4, __uint_as_float(xr[j].w));
         }
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            // widen the eight BF16 weights to FP32 (exact) on the way to shared memory
+        for (int j = 0; j < NW; ++j) {
             const uint32_t a = wb + ws_off[j];
-            sts32(a, up_lo(wr[j].x));
-            sts32(a + kPitch * 4, up_hi(wr[j].x));
-            sts32(a + 2 * kPitch * 4, up_lo(wr[j].y));
-            sts32(a + 3 * kPitch * 4, up_hi(wr[j].y));
-            sts32(a + 4 * kPitch * 4, up_lo(wr[j].z));
-            sts32(a + 5 * kPitch * 4, up_hi(wr[j].z));
-            sts32(a + 6 * kPitch * 4, up_lo(wr[j].w));
-            sts32(a + 7 * kPitch * 4, up_hi(wr[j].w));
+            if constexpr (WF == 2) {
+                sts32(a, __uint_as_float(wr[j].x));
+                sts32(a + kPitch * 4, __uint_as_float(wr[j].y));
+                sts32(a + 2 * kPitch * 4, __uint_as_float(wr[j].z));
+                sts32(a + 3 * kPitch * 4, __uint_as_float(wr[j].w));
+            } else {
+                // widen the eight 16-bit weights to FP32 (exact) on the way to shared memory
+                sts32(a, up16_lo<WF>(wr[j].x));
+                sts32(a + kPitch * 4, up16_hi<WF>(wr[j].x));
+                sts32(a + 2 * kPitch * 4, up16_lo<WF>(wr[j].y));
+                sts32(a + 3 * kPitch * 4, up16_hi<WF>(wr[j].y));
+                sts32(a + 4 * kPitch * 4, up16_lo<WF>(wr[j].z));
+                sts32(a + 5 * kPitch * 4, up16_hi<WF>(wr[j].z));
+                sts32(a + 6 * kPitch * 4, up16_lo<WF>(wr[j].w));
+                sts32(a + 7 * kPitch * 4, up16_hi<WF>(wr[j].w));
+            }
         }
     };
 
@@ -214,11 +227,14 @@ prefill_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W, cons
 
 }  // namespace
 
-cudaError_t launch_prefill(const LaunchArgs& a)
+namespace {
+
+template <int WF>
+cudaError_t launch_prefill_t(const LaunchArgs& a)
 {
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(prefill_kernel<WF>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -226,13 +242,25 @@ cudaError_t launch_prefill(const LaunchArgs& a)
     const long long units = (long long)tiles_m * tiles_n * a.S;
     if (units > 0x7fffffffLL) return cudaErrorInvalidValue;
     const int direct = (a.S == 1);
-    prefill_kernel<<<(unsigned)units, kThreads, kSmemBytes, a.stream>>>(a.x, a.W, a.b, direct ? a.y : a.partials, (int)a.M,
-                                                                        (int)a.N, (int)a.K, (int)a.seg_len, a.S, direct,
-                                                                        tiles_m, tiles_n);
+    prefill_kernel<WF><<<(unsigned)units, kThreads, kSmemBytes, a.stream>>>(
+        a.x, static_cast<const typename WeightElem<WF>::type*>(a.W), a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N,
+        (int)a.K, (int)a.seg_len, a.S, direct, tiles_m, tiles_n);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (!direct) return launch_combine(a);
     return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_prefill(const LaunchArgs& a)
+{
+    switch (a.wfmt) {
+    case DET_WEIGHT_BF16: return launch_prefill_t<0>(a);
+    case DET_WEIGHT_FP16: return launch_prefill_t<1>(a);
+    case DET_WEIGHT_FP32: return launch_prefill_t<2>(a);
+    default: return cudaErrorInvalidValue;
+    }
 }
 
 }  // namespace detlin

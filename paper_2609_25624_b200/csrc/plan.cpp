@@ -70,6 +70,7 @@ det_status_t fill_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* o
     p.seg_len = seg_len;
     p.S = (int32_t)S;
     p.order_version = kOrderVersion;
+    p.weight_format = DET_WEIGHT_BF16;
     p.kernel = (K % 8 == 0) ? (p.bucket == 0 ? kKernelDecode : kKernelPrefill) : kKernelGeneric;
     p.workspace_bytes = p.S > 1 ? (uint64_t)4 * (uint64_t)p.S * (uint64_t)M * (uint64_t)N : 0;
     *out = p;

@@ -43,6 +43,38 @@ def make_case(M: int, N: int, K: int, seed=None, bias: bool = True):
     return x, W, b
 
 
+#: torch dtype that carries each weight format
+WEIGHT_DTYPES = {"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}
+
+
+def make_case_w(M: int, N: int, K: int, wfmt: str, seed=None, bias: bool = True):
+    """make_case with the weights stored as "bf16", "fp16" or "fp32": the same FP32 draws, rounded to
+    nearest even into the 16-bit formats (about 0.2 % of the FP16 weights are then subnormal) or
+    kept as drawn for FP32."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(shape_seed(M, N, K) if seed is None else int(seed))
+    W = (0.02 * torch.randn(N, K, dtype=torch.float32, generator=g)).to(WEIGHT_DTYPES[wfmt])
+    x = torch.randn(M, K, dtype=torch.float32, generator=g)
+    b = 0.01 * torch.randn(N, dtype=torch.float32, generator=g) if bias else None
+    return x, W, b
+
+
+def weight_format_of(W: torch.Tensor) -> str:
+    for name, dt in WEIGHT_DTYPES.items():
+        if W.dtype == dt:
+            return name
+    raise ValueError(f"no weight format for dtype {W.dtype}")
+
+
+def weight_bits(W: torch.Tensor) -> np.ndarray:
+    """Weight tensor -> numpy array of its stored elements: uint16 bit patterns for the 16-bit
+    formats, float32 for FP32 (same memory layout)."""
+    if W.dtype == torch.float32:
+        return W.contiguous().numpy()
+    assert W.dtype in (torch.bfloat16, torch.float16)
+    return W.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
 def make_weight(N: int, K: int, seed: int):
     """One BF16 weight matrix [N,K] ~ N(0, 0.02^2) (for the multi-layer stack)."""
     g = torch.Generator(device="cpu")

@@ -13,13 +13,14 @@ def to_dev(t):
 
 
 def run_gpu(x, W, b, kernel=None, variant=0, max_blocks=0, stream=None, y_fill=float("nan")):
-    """x [M,K] f32, W [N,K] bf16, b [N] f32 or None (CPU or CUDA tensors) -> y as numpy float32 [M,N].
+    """x [M,K] f32, W [N,K] bf16 / fp16 / fp32 (the plan's weight format follows the dtype), b [N] f32 or
+    None (CPU or CUDA tensors) -> y as numpy float32 [M,N].
     The output buffer is pre-filled with NaN so that an element the kernel never wrote is caught."""
     M, K = x.shape
     N = W.shape[0]
     xd, Wd, bd = x.cuda(), W.cuda(), to_dev(b)
     y = torch.full((M, N), y_fill, dtype=torch.float32, device="cuda")
-    plan = B.det_linear_plan(M, N, K)
+    plan = B.det_linear_plan_w(M, N, K, inputs.weight_format_of(W))
     try:
         if kernel is not None:
             B.det_test_plan_force_kernel(plan, kernel)
@@ -37,7 +38,8 @@ def run_gpu(x, W, b, kernel=None, variant=0, max_blocks=0, stream=None, y_fill=f
 
 def oracle_y(x, W, b):
     from oracle import oracle
-    return oracle.linear(x.numpy(), inputs.bf16_bits(W), None if b is None else b.numpy())
+    return oracle.linear(x.numpy(), inputs.weight_bits(W), None if b is None else b.numpy(),
+                         wfmt=inputs.weight_format_of(W))
 
 
 def assert_bits_equal(got, want, what=""):
