@@ -315,6 +315,7 @@ def run_own(args, world, rank, local):
         line["prefill"] = prefill_table(B, dev, st, fp32_peak)
         line["lm_head"] = lm_head_table(B, dev, st, hbm_peak, fp32_peak)
         line["layercast_style_reference"] = layercast_table(work, st, line["per_case"])
+        line["weight_formats"] = weight_format_table(B, dev, st, hbm_peak, fp32_peak)
         line["cpu_baseline"] = cpu_baseline(work)
         for w in work:                       # free the sweep's 2.2 GB before the 15 GB stack
             w["plan"].close()
@@ -450,6 +451,46 @@ def lm_head_table(B, dev, st, hbm_peak, fp32_peak):
         rows.append({"M": M, "us_linear_plus_argmax": ms * 1e3, "weight_gbs": wbytes / ms / 1e6,
                      "pct_hbm": 100 * wbytes / ms / 1e6 / hbm_peak, "tflops": 2 * M * N * K / ms / 1e9,
                      "pct_fp32": 100 * 2 * M * N * K / ms / 1e9 / fp32_peak})
+    return rows
+
+
+def weight_format_table(B, dev, st, hbm_peak, fp32_peak):
+    """The same calls with the weight matrix stored as BF16, FP16 or FP32 (the order and the output
+    rounding steps are the same; only the bytes streamed and the widening differ).  Decode rows cycle
+    through clones of W totalling >= 512 MB (cold weights); the prefill row is compute-bound."""
+    name, K, N = inputs.LLAMA3_8B_LAYER[2]           # gate_up 4096 -> 28672
+    rows = []
+    for wfmt in ("bf16", "fp16", "fp32"):
+        eb = 4 if wfmt == "fp32" else 2
+        _, W0, b = inputs.make_case_w(1, N, K, wfmt)
+        W0, bd = W0.to(dev), b.to(dev)
+        wbytes = eb * N * K
+        R = max(2, -(-(512 << 20) // wbytes))
+        Ws = [W0] + [W0.clone() for _ in range(R - 1)]
+        for M in (1, 8, 32, 512):
+            g = torch.Generator().manual_seed(inputs.shape_seed(M, N, K))
+            x = torch.randn(M, K, generator=g).to(dev)
+            y = torch.empty(M, N, dtype=torch.float32, device=dev)
+            plans = [B.det_linear_plan_w(M, N, K, wfmt) for _ in range(R)]
+            reps = R * max(1, 8 // R) if M <= 64 else R
+
+            def call():
+                for i in range(reps):
+                    B.det_linear_run(plans[i % R], x, Ws[i % R], bd, y)
+            with torch.cuda.stream(st):
+                call()
+                torch.cuda.synchronize()
+            ms = time_graph(call, 3, st) / reps
+            for p in plans:
+                B.det_linear_plan_check(p)
+                p.close()
+            t_hbm = wbytes / (hbm_peak * 1e9)
+            t_fma = 2 * M * N * K / (fp32_peak * 1e12)
+            rows.append({"weights": wfmt, "name": name, "M": M, "N": N, "K": K, "us": ms * 1e3,
+                         "weight_gbs": wbytes / ms / 1e6, "tflops": 2 * M * N * K / ms / 1e9,
+                         "bound": "hbm" if t_hbm >= t_fma else "fp32",
+                         "pct_of_roofline": 100 * max(t_hbm, t_fma) / (ms * 1e-3)})
+        del Ws
     return rows
 
 

@@ -14,6 +14,8 @@ static const DecodeEntry kEntries0[] = {
     DEC(1, 1, 8, 4, 128, 6, 1),
     DEC(1, 1, 8, 2, 256, 4, 1),
     DEC(1, 1, 2, 4, 256, 8, 1),
+    DEC(1, 1, 8, 4, 256, 3, 1),
+    DEC(1, 1, 16, 2, 128, 4, 1),
 };
 #else
 static const DecodeEntry kEntries0[] = {
@@ -32,6 +34,8 @@ static const DecodeEntry kEntries1[] = {
     DEC(2, 1, 8, 4, 128, 6, 1),
     DEC(2, 1, 8, 2, 256, 4, 1),
     DEC(2, 1, 2, 4, 256, 8, 1),
+    DEC(2, 1, 8, 4, 256, 3, 1),
+    DEC(2, 1, 16, 2, 128, 4, 1),
 };
 #else
 static const DecodeEntry kEntries1[] = {
@@ -51,6 +55,8 @@ static const DecodeEntry kEntries2[] = {
     DEC(4, 1, 6, 4, 128, 5, 1),
     DEC(4, 1, 14, 4, 128, 3, 1),
     DEC(4, 1, 8, 2, 128, 6, 1),
+    DEC(4, 1, 8, 4, 256, 3, 1),
+    DEC(4, 1, 6, 4, 256, 4, 1),
 };
 #else
 static const DecodeEntry kEntries2[] = {

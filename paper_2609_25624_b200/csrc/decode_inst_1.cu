@@ -17,6 +17,9 @@ static const DecodeEntry kEntries3[] = {
     DEC(8, 1, 12, 4, 128, 3, 4),
     DEC(8, 1, 14, 4, 128, 3, 4),
     DEC(8, 1, 8, 2, 128, 6, 1),
+    DEC(8, 1, 8, 4, 256, 3, 1),
+    DEC(8, 1, 12, 4, 256, 3, 4),
+    DEC(8, 1, 14, 4, 256, 3, 4),
 };
 #else
 static const DecodeEntry kEntries3[] = {

@@ -15,6 +15,9 @@ static const DecodeEntry kEntries4[] = {
     DEC(8, 2, 10, 4, 128, 3, 4),
     DEC(8, 2, 12, 4, 128, 3, 4),
     DEC(8, 2, 14, 4, 128, 3, 4),
+    DEC(8, 2, 8, 4, 256, 3, 4),
+    DEC(8, 2, 12, 4, 256, 3, 4),
+    DEC(8, 2, 14, 4, 256, 3, 4),
 };
 #else
 static const DecodeEntry kEntries4[] = {

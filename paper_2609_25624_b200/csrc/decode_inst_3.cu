@@ -15,6 +15,10 @@ static const DecodeEntry kEntries5[] = {
     DEC(8, 4, 12, 2, 128, 3, 4),
     DEC(8, 4, 14, 2, 128, 3, 4),
     DEC(8, 4, 16, 2, 128, 3, 4),
+    DEC(8, 4, 8, 2, 256, 3, 4),
+    DEC(8, 4, 12, 2, 256, 3, 4),
+    DEC(8, 4, 14, 2, 256, 3, 4),
+    DEC(8, 4, 16, 2, 256, 3, 4),
 };
 #else
 static const DecodeEntry kEntries5[] = {
