@@ -313,6 +313,7 @@ def run_own(args, world, rank, local):
     if not args.no_extras:
         line["per_case"] = per_case_table(B, work, st, hbm_peak, fp32_peak)
         line["prefill"] = prefill_table(B, dev, st, fp32_peak)
+        line["mid_bucket"] = mid_bucket_table(B, dev, st, fp32_peak)
         line["lm_head"] = lm_head_table(B, dev, st, hbm_peak, fp32_peak)
         line["layercast_style_reference"] = layercast_table(work, st, line["per_case"])
         line["weight_formats"] = weight_format_table(B, dev, st, hbm_peak, fp32_peak)
@@ -422,6 +423,32 @@ def prefill_table(B, dev, st, fp32_peak):
     return {"fp32_peak_tflops": fp32_peak, "peak_source": "148 SMs x 128 lanes x 2 x 1965 MHz (derived)",
             "aggregate_tflops": total_flops / total_s / 1e12, "aggregate_pct_fp32_peak": 100 * total_flops / total_s / 1e12 / fp32_peak,
             "cases": rows}
+
+
+def mid_bucket_table(B, dev, st, fp32_peak):
+    """Batch sizes between the decode bucket and a full 128-row prefill tile (and just above a
+    multiple of 128): the prefill kernel picks the tile height (80 .. 128 rows) that pads least."""
+    rows = []
+    for (name, K, N) in inputs.PREFILL_SHAPES:
+        W = None
+        for M in (72, 96, 160):
+            x, Wc, b = inputs.make_case(M, N, K)
+            if W is None:
+                W = Wc.to(dev)
+            xd, bd = x.to(dev), b.to(dev)
+            y = torch.empty(M, N, dtype=torch.float32, device=dev)
+            plan = B.det_linear_plan(M, N, K)
+            with torch.cuda.stream(st):
+                B.det_linear_run(plan, xd, W, bd, y)
+                torch.cuda.synchronize()
+            ms = time_graph(lambda: B.det_linear_run(plan, xd, W, bd, y), 3, st)
+            B.det_linear_plan_check(plan)
+            tile = B.det_linear_plan_describe(plan)["prefill_tile"]
+            plan.close()
+            tf = 2 * M * N * K / ms / 1e9
+            rows.append({"name": name, "M": M, "N": N, "K": K, "tile_rows": tile["bm"], "us": ms * 1e3, "tflops": tf,
+                         "pct_fp32_peak": 100 * tf / fp32_peak})
+    return rows
 
 
 def lm_head_table(B, dev, st, hbm_peak, fp32_peak):

@@ -259,13 +259,18 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
             snprintf(tiling, sizeof tiling, "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"kc\": %d, \"stages\": %d}", c.mt,
                      c.wm, c.rt, c.wr, c.kc, c.stages);
     }
+    char ptile[64] = "null";
+    if (p.kernel == kKernelPrefill) {
+        const int tr = (plan->variant >= 5 && plan->variant <= 8) ? plan->variant : prefill_rows_per_thread(p.M);
+        snprintf(ptile, sizeof ptile, "{\"bm\": %d, \"bn\": 128, \"bk\": 32}", 16 * tr);
+    }
     int w = snprintf(buf, n,
                      "{\"M\": %lld, \"N\": %lld, \"K\": %lld, \"bucket\": \"%s\", \"V\": %d, \"L\": %d, \"P\": %d, "
                      "\"seg_len\": %lld, \"S\": %d, \"order_version\": %d, \"kernel\": \"%s\", \"workspace_bytes\": %llu, "
-                     "\"weight_format\": \"%s\", \"decode_tiling\": %s}",
+                     "\"weight_format\": \"%s\", \"decode_tiling\": %s, \"prefill_tile\": %s}",
                      (long long)p.M, (long long)p.N, (long long)p.K, p.bucket == 0 ? "decode" : "prefill", p.V, p.L, p.P,
                      (long long)p.seg_len, p.S, p.order_version, kn[p.kernel], (unsigned long long)p.workspace_bytes,
-                     p.weight_format == DET_WEIGHT_FP32 ? "fp32" : p.weight_format == DET_WEIGHT_FP16 ? "fp16" : "bf16", tiling);
+                     p.weight_format == DET_WEIGHT_FP32 ? "fp32" : p.weight_format == DET_WEIGHT_FP16 ? "fp16" : "bf16", tiling, ptile);
     if (w < 0 || (size_t)w >= n) { set_error("describe: buffer too small (%d bytes needed)", w + 1); return DET_ERR_INVALID_ARG; }
     return DET_OK;
 }
@@ -324,6 +329,9 @@ det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
             set_error("set_variant: the decode kernel has fewer than %d tilings for this batch size", variant);
             return DET_ERR_INVALID_ARG;
         }
+    } else if (variant != 0 && (variant < 5 || variant > 8)) {
+        set_error("set_variant: the prefill kernel takes 0 (automatic) or 5 .. 8 rows per thread");
+        return DET_ERR_INVALID_ARG;
     }
     plan->variant = variant;
     return DET_OK;

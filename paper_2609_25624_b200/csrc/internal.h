@@ -46,6 +46,8 @@ cudaError_t launch_generic(const LaunchArgs& a, int bucket);
 cudaError_t launch_combine(const LaunchArgs& a);
 cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x);
 cudaError_t launch_prefill(const LaunchArgs& a);
+// rows per thread (tile height = 16 x this) the prefill kernel uses for batch size M; schedule only
+int prefill_rows_per_thread(int64_t M);
 cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cudaStream_t stream);
 
 // Decode-kernel tiling chosen for a shape (numerically inert); used by the host to build the

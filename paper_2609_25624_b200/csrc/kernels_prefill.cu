@@ -9,7 +9,8 @@
 // bits.  Measured on B200 this loop sustains more than the scalar-FMA form of the same tile because
 // the packed instruction leaves every other issue slot free for the shared-memory loads.
 //
-// Schedule (numerically inert): 128 x 128 output tile per block, 256 threads, 8 x 8 outputs per
+// Schedule (numerically inert): 128 x 128 output tile per block (16 TR x 128 with TR = 5 .. 7 rows per
+// thread when that pads the batch less), 256 threads, 8 x 8 outputs per
 // thread (4 column pairs), two blocks per SM, K walked in slabs of 32 with two slab buffers.  Both
 // operands are staged k-major ([k][m] and [k][n]) so that a thread reads its eight x values and its
 // eight weights of one k with four 16-byte loads.  16-bit weights are widened to FP32 once per block
@@ -22,7 +23,7 @@ namespace detlin {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 32;
+constexpr int BN = 128, BK = 32;
 constexpr int kThreads = 256;
 constexpr int kPitch = 132;                         // floats per k row: 128 + 4 keeps 16-byte alignment
 constexpr int kTileFloats = BK * kPitch;
@@ -45,8 +46,26 @@ __device__ __forceinline__ uint4 ldg128_nc(const void* p)
     return v;
 }
 
+// n consecutive floats from shared memory (n <= 4; the address is 4 n-byte aligned for n = 1, 2, 4)
+template <int N_>
+__device__ __forceinline__ void lds_floats(uint32_t addr, float* v)
+{
+    if constexpr (N_ == 4) {
+        const float4 t = lds128(addr);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else if constexpr (N_ == 2) {
+        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v[0]), "=f"(v[1]) : "r"(addr));
+    } else {
+#pragma unroll
+        for (int i = 0; i < N_; ++i) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v[i]) : "r"(addr + 4 * i));
+    }
+}
+
 // WF: weight format (0 BF16, 1 FP16: octets of 16-bit weights; 2 FP32: quads, staged like x)
-template <int WF>
+// TR: output rows per thread (5 .. 8); the block tile is BM = 16 TR rows by 128 columns.  The row count
+//     of the tile is schedule only: batch sizes between two multiples of 128 (the "mid bucket"
+//     65 <= M < 128 in particular) get the tile height that wastes the fewest rows.
+template <int WF, int TR>
 __global__ void __launch_bounds__(kThreads, 2)
 prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type* __restrict__ W, const float* __restrict__ bias,
                float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct, int tiles_m, int tiles_n)
@@ -56,6 +75,9 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
     // buffer b: x tile at smem + b*2*T, w tile at smem + (b*2+1)*T, T = kTileFloats*4 bytes
     constexpr uint32_t T = kTileFloats * 4;
 
+    constexpr int BM = 16 * TR;
+    constexpr int TB = TR - 4;                       // rows of a thread in the upper group (1 .. 4)
+    constexpr int XP = (BM * 8 + 255) / 256;         // 16-byte pieces of x per thread and slab
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
 
@@ -70,23 +92,23 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
     const int k_hi = min(K, k_lo + seg_len);
 
     // ---- staging assignment (global rows are k-contiguous, shared tiles are k-major: a transpose) ----
-    // x tile: 128 rows x 8 quads (4 floats = 16 bytes).  Piece p = tid + 256 j: half o = p & 1,
-    //   row r = (p >> 1) & 127, quad q = 2 * (p >> 8) + o.  Two neighbouring lanes read one 32-byte
+    // x tile: BM rows x 8 quads (4 floats = 16 bytes).  Piece p = tid + 256 j: half o = p & 1,
+    //   row r = (p >> 1) mod BM, quad q = 2 * ((p >> 1) / BM) + o.  Two neighbouring lanes read one 32-byte
     //   sector; the four scalar stores of a lane go to k rows 4q .. 4q+3, conflict-free across the warp
     //   (bank = 16 o + 4 e + r mod 32 over 16 consecutive r and o in {0, 1}).
     // w tile: 128 rows x 4 octets (8 BF16 = 16 bytes).  Piece p = tid + 256 j: half o = p & 1,
     //   row r = (p >> 1) & 127, octet c = 2 * (p >> 8) + o; eight scalar stores to k rows 8c .. 8c+7
     //   (two-way bank conflicts between the two halves; 16 stores per thread and slab).
-    const float* xg[4];
-    uint32_t xs_off[4];
-    int xk[4];
-    bool xok[4];
+    const float* xg[XP];
+    uint32_t xs_off[XP];
+    int xk[XP];
+    bool xok[XP];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < XP; ++j) {
         const int p = tid + 256 * j;
-        const int o = p & 1, r = (p >> 1) & 127, q = 2 * (p >> 8) + o;
+        const int o = p & 1, r = (p >> 1) % BM, q = 2 * ((p >> 1) / BM) + o;
         const int m = m0 + r;
-        xok[j] = m < M;
+        xok[j] = m < M && p < BM * 8;
         xk[j] = q * 4;
         xg[j] = x + (long long)(xok[j] ? m : 0) * K + q * 4;
         xs_off[j] = (uint32_t)((q * 4) * kPitch + r) * 4;
@@ -109,13 +131,13 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
         ws_off[j] = (uint32_t)((c * WE) * kPitch + r) * 4;
     }
 
-    uint4 xr[4];
+    uint4 xr[XP];
     uint4 wr[NW];
     auto load_slab = [&](int k0) {
         // the row pitch is a whole number of 16-byte pieces: a piece of weights / a quad of activations is
         // entirely inside or outside [.., k_hi)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < XP; ++j) {
             if (xok[j] && k0 + xk[j] < k_hi) xr[j] = ldg128_nc(xg[j] + k0);
             else xr[j] = make_uint4(0u, 0u, 0u, 0u);
         }
@@ -128,7 +150,8 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
     auto store_slab = [&](int buf) {
         const uint32_t xb = smem + (uint32_t)(buf * 2) * T, wb = xb + T;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < XP; ++j) {
+            if ((BM * 8) % 256 != 0 && tid + 256 * j >= BM * 8) continue;   // odd TR: the last round is half empty
             const uint32_t a = xb + xs_off[j];
             sts32(a, __uint_as_float(xr[j].x));
             sts32(a + kPitch * 4, __uint_as_float(xr[j].y));
@@ -157,11 +180,11 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
         }
     };
 
-    // acc[i][j]: rows m0 + (i < 4 ? 4 ty + i : 64 + 4 ty + i - 4); column pair j:
+    // acc[i][j]: rows m0 + (i < 4 ? 4 ty + i : 64 + TB ty + i - 4); column pair j:
     //   (n0 + 4 tx + 2 j, +1) for j < 2, (n0 + 64 + 4 tx + 2 (j - 2), +1) for j >= 2
-    float2 acc[8][4];
+    float2 acc[TR][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < TR; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
 
@@ -174,20 +197,21 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
         const bool more = k0 + BK < k_hi;
         if (more) load_slab(k0 + BK);
         const uint32_t xb = smem + (uint32_t)(buf * 2) * T + (uint32_t)(ty * 4) * 4;
+        const uint32_t xb2 = xb + (uint32_t)(64 + ty * (TB - 4)) * 4;     // upper group: rows 64 + TB ty ..
         const uint32_t wb = smem + (uint32_t)(buf * 2 + 1) * T + (uint32_t)(tx * 4) * 4;
         // k beyond the end of the segment is skipped, not zero-filled
         const int nk = min(BK, k_hi - k0);
 #pragma unroll 4
         for (int kk = 0; kk < nk; ++kk) {
-            const float4 xa = lds128(xb + (uint32_t)(kk * kPitch) * 4);
-            const float4 xc = lds128(xb + (uint32_t)(kk * kPitch + 64) * 4);
+            float xv[TR];
+            lds_floats<4>(xb + (uint32_t)(kk * kPitch) * 4, xv);
+            lds_floats<TB>(xb2 + (uint32_t)(kk * kPitch) * 4, xv + 4);
             const float4 wa = lds128(wb + (uint32_t)(kk * kPitch) * 4);
             const float4 wc = lds128(wb + (uint32_t)(kk * kPitch + 64) * 4);
-            const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xc.x, xc.y, xc.z, xc.w};
             const float2 wp[4] = {make_float2(wa.x, wa.y), make_float2(wa.z, wa.w), make_float2(wc.x, wc.y),
                                   make_float2(wc.z, wc.w)};
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < TR; ++i) {
                 const float2 x2 = make_float2(xv[i], xv[i]);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) acc[i][j] = __ffma2_rn(x2, wp[j], acc[i][j]);
@@ -201,8 +225,8 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
     // ---- epilogue: bias (direct) or the segment's partial ----
     const bool vec_ok = (N % 4 == 0);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int m = m0 + (i < 4 ? 4 * ty + i : 64 + 4 * ty + (i - 4));
+    for (int i = 0; i < TR; ++i) {
+        const int m = m0 + (i < 4 ? 4 * ty + i : 64 + TB * ty + (i - 4));
         if (m >= M) continue;
         float* orow = direct ? out + (long long)m * N : out + ((long long)s * M + m) * N;
 #pragma unroll
@@ -229,12 +253,13 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
 
 namespace {
 
-template <int WF>
+template <int WF, int TR>
 cudaError_t launch_prefill_t(const LaunchArgs& a)
 {
+    constexpr int BM = 16 * TR;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_kernel<WF>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(prefill_kernel<WF, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -242,7 +267,7 @@ cudaError_t launch_prefill_t(const LaunchArgs& a)
     const long long units = (long long)tiles_m * tiles_n * a.S;
     if (units > 0x7fffffffLL) return cudaErrorInvalidValue;
     const int direct = (a.S == 1);
-    prefill_kernel<WF><<<(unsigned)units, kThreads, kSmemBytes, a.stream>>>(
+    prefill_kernel<WF, TR><<<(unsigned)units, kThreads, kSmemBytes, a.stream>>>(
         a.x, static_cast<const typename WeightElem<WF>::type*>(a.W), a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N,
         (int)a.K, (int)a.seg_len, a.S, direct, tiles_m, tiles_n);
     cudaError_t e = cudaGetLastError();
@@ -251,14 +276,39 @@ cudaError_t launch_prefill_t(const LaunchArgs& a)
     return cudaSuccess;
 }
 
+template <int WF>
+cudaError_t launch_prefill_f(const LaunchArgs& a, int tr)
+{
+    switch (tr) {
+    case 5: return launch_prefill_t<WF, 5>(a);
+    case 6: return launch_prefill_t<WF, 6>(a);
+    case 7: return launch_prefill_t<WF, 7>(a);
+    default: return launch_prefill_t<WF, 8>(a);
+    }
+}
+
 }  // namespace
+
+// Rows per thread (tile height 16 TR) that pads the batch least; ties go to the taller tile.  Schedule
+// only: every height gives the same bits.  a.variant 5 .. 8 forces a height (tests).
+int prefill_rows_per_thread(int64_t M)
+{
+    int best = 8;
+    int64_t best_rows = ((M + 127) / 128) * 128;
+    for (int tr = 7; tr >= 5; --tr) {
+        const int64_t bm = 16 * tr, rows = ((M + bm - 1) / bm) * bm;
+        if (rows < best_rows) { best_rows = rows; best = tr; }
+    }
+    return best;
+}
 
 cudaError_t launch_prefill(const LaunchArgs& a)
 {
+    const int tr = (a.variant >= 5 && a.variant <= 8) ? a.variant : prefill_rows_per_thread(a.M);
     switch (a.wfmt) {
-    case DET_WEIGHT_BF16: return launch_prefill_t<0>(a);
-    case DET_WEIGHT_FP16: return launch_prefill_t<1>(a);
-    case DET_WEIGHT_FP32: return launch_prefill_t<2>(a);
+    case DET_WEIGHT_BF16: return launch_prefill_f<0>(a, tr);
+    case DET_WEIGHT_FP16: return launch_prefill_f<1>(a, tr);
+    case DET_WEIGHT_FP32: return launch_prefill_f<2>(a, tr);
     default: return cudaErrorInvalidValue;
     }
 }

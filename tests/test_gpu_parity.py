@@ -181,3 +181,33 @@ def test_bad_arguments_are_rejected():
     with pytest.raises(B.DetLinearError):
         B.det_test_plan_force_kernel(plan, KERNEL_PREFILL)
     plan.close()
+
+
+MID_BUCKET = [(65, 130, 520), (72, 256, 1024), (80, 200, 1000), (96, 144, 2048), (100, 1000, 1000), (112, 128, 512),
+              (127, 129, 264), (130, 64, 512), (200, 72, 4096), (300, 136, 776)]
+
+
+@pytest.mark.parametrize("M,N,K", MID_BUCKET)
+def test_prefill_tile_heights_bit_exact(M, N, K):
+    """The prefill tile height (80, 96, 112 or 128 rows) is schedule only: every height, forced or
+    chosen automatically, reproduces the oracle's bits (the mid bucket 65 <= M < 128 and batch
+    sizes just above a multiple of 128 get a shorter tile)."""
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    for variant in (0, 5, 6, 7, 8):
+        assert_bits_equal(run_gpu(x, W, b, kernel=KERNEL_PREFILL, variant=variant), want, f"rows per thread {variant}")
+
+
+def test_prefill_tile_choice():
+    for M, bm in ((65, 80), (72, 80), (81, 96), (100, 112), (113, 128), (128, 128), (130, 80), (200, 112), (512, 128),
+                  (2048, 128), (257, 96)):
+        plan = B.det_linear_plan(M, 256, 512)
+        d = B.det_linear_plan_describe(plan)
+        plan.close()
+        assert d["kernel"] == "prefill" and d["prefill_tile"]["bm"] == bm, (M, d)
+        padded = -(-M // bm) * bm
+        assert all(padded <= -(-M // h) * h for h in (80, 96, 112, 128)), (M, bm)
+    plan = B.det_linear_plan(100, 256, 512)
+    with pytest.raises(B.DetLinearError):
+        B.det_test_plan_set_variant(plan, 3)
+    plan.close()
