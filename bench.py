@@ -317,6 +317,7 @@ def run_own(args, world, rank, local):
         line["lm_head"] = lm_head_table(B, dev, st, hbm_peak, fp32_peak)
         line["layercast_style_reference"] = layercast_table(work, st, line["per_case"])
         line["weight_formats"] = weight_format_table(B, dev, st, hbm_peak, fp32_peak)
+        line["column_shards"] = shard_table(B, dev, st, hbm_peak)
         line["cpu_baseline"] = cpu_baseline(work)
         for w in work:                       # free the sweep's 2.2 GB before the 15 GB stack
             w["plan"].close()
@@ -448,6 +449,40 @@ def mid_bucket_table(B, dev, st, fp32_peak):
             tf = 2 * M * N * K / ms / 1e9
             rows.append({"name": name, "M": M, "N": N, "K": K, "tile_rows": tile["bm"], "us": ms * 1e3, "tflops": tf,
                          "pct_fp32_peak": 100 * tf / fp32_peak})
+    return rows
+
+
+def shard_table(B, dev, st, hbm_peak):
+    """What one rank of a column-parallel group of `world` GPUs runs: the first shard of gate_up and
+    down at M = 1 and 8 (single GPU here, so only the per-rank kernel time is measured; the all-gather
+    is not).  Cold weights: the graph cycles through clones of the shard totalling >= 512 MB."""
+    from paper_2609_25624_b200.sharded import shard_range
+    rows = []
+    for (name, K, N) in (inputs.LLAMA3_8B_LAYER[2], inputs.LLAMA3_8B_LAYER[3]):
+        for world in (2, 8):
+            n0, cnt = shard_range(N, 0, world)
+            Wc = inputs.make_weight(cnt, K, inputs.named_seed(f"shard.{name}.{world}")).to(dev)
+            wbytes = 2 * cnt * K
+            R = max(2, -(-(512 << 20) // wbytes))
+            Ws = [Wc] + [Wc.clone() for _ in range(R - 1)]
+            for M in (1, 8):
+                x = torch.randn(M, K, generator=torch.Generator().manual_seed(M)).to(dev)
+                y = torch.empty(M, cnt, dtype=torch.float32, device=dev)
+                plans = [B.det_linear_plan_shard(M, N, K, n0, cnt, cnt) for _ in range(R)]
+
+                def call():
+                    for i in range(R):
+                        B.det_linear_run_shard(plans[i], x, Ws[i], None, y)
+                with torch.cuda.stream(st):
+                    call()
+                    torch.cuda.synchronize()
+                ms = time_graph(call, 3, st) / R
+                for p in plans:
+                    B.det_linear_plan_check(p)
+                    p.close()
+                rows.append({"name": name, "world": world, "M": M, "n_count": cnt, "K": K, "us_per_rank": ms * 1e3,
+                             "weight_gbs_per_rank": wbytes / ms / 1e6, "pct_hbm": 100 * wbytes / ms / 1e6 / hbm_peak})
+            del Ws
     return rows
 
 

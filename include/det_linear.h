@@ -98,6 +98,26 @@ DET_API det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K);
 DET_API det_linear_plan_t* det_linear_plan_w(int64_t M, int64_t N, int64_t K, int32_t wfmt);
 
 /*
+ * Plan for ONE COLUMN SHARD of a layer: outputs n_begin .. n_begin + n_count - 1 of y[M,N] (tensor
+ * parallelism over the output dimension).  Every output depends on one weight row only, and the
+ * order parameters are those of the whole layer (M, N, K) -- the split factor is evaluated on the
+ * global N -- so a shard's outputs carry the same bits as the same columns computed by
+ * det_linear_plan(M, N, K) on one GPU, whatever the number of shards.  The paper runs on a single
+ * GPU; this is the column-parallel extension its reduction order allows without any change.
+ * With such a plan det_linear_run_w takes
+ *   W : the shard's rows, [n_count, K] row-major (element (0,0) = weight row n_begin of the layer)
+ *   b : the shard's n_count bias values, or NULL
+ *   y : address of the shard's first column inside a row-major matrix with row pitch `ldy` floats
+ *       (ldy = N writes in place into the full [M,N] output, ldy = n_count gives a compact block)
+ * The fast kernels need y 16-byte aligned (and ldy % 4 == 0 in the prefill bucket); otherwise the
+ * generic kernels run.  Requires 0 <= n_begin, 1 <= n_count, n_begin + n_count <= N, ldy >= n_count.
+ * det_linear_plan_params / get_params report the layer's N; workspace_bytes is the shard's.
+ * det_linear_run_host* reject shard plans.  The all-gather of the shards is the caller's.
+ */
+DET_API det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K, int64_t n_begin, int64_t n_count,
+                                                 int64_t ldy, int32_t wfmt);
+
+/*
  * Enqueue the computation on `stream` (a cudaStream_t; NULL = the legacy default stream) and
  * return without synchronising.  Eq. 2 with the order above; split-K partials, if any, are
  * combined by a second fixed-order pass (R3), never by atomics.

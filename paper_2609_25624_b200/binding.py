@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.det_linear_plan.restype = p
         L.det_linear_plan_w.argtypes = [i64, i64, i64, ctypes.c_int32]
         L.det_linear_plan_w.restype = p
+        L.det_linear_plan_shard.argtypes = [i64, i64, i64, i64, i64, i64, ctypes.c_int32]
+        L.det_linear_plan_shard.restype = p
         L.det_linear_run.argtypes = [p, p, p, p, p, p]
         L.det_linear_run.restype = i32
         L.det_linear_run_w.argtypes = [p, p, p, p, p, p]
@@ -130,11 +132,15 @@ WEIGHT_FORMATS = {"bf16": DET_WEIGHT_BF16, "fp16": DET_WEIGHT_FP16, "fp32": DET_
 class Plan:
     """Owner of a det_linear_plan_t*."""
 
-    def __init__(self, M: int, N: int, K: int, wfmt: int = DET_WEIGHT_BF16):
+    def __init__(self, M: int, N: int, K: int, wfmt: int = DET_WEIGHT_BF16, shard=None):
+        """shard = (n_begin, n_count, ldy) makes a column-shard plan (det_linear_plan_shard)."""
         self.M, self.N, self.K = int(M), int(N), int(K)
         self.wfmt = WEIGHT_FORMATS.get(wfmt, wfmt) if isinstance(wfmt, str) else int(wfmt)
         self.w_dtype = WEIGHT_DTYPES.get(self.wfmt, torch.bfloat16)
-        if self.wfmt == DET_WEIGHT_BF16:
+        self.shard = None if shard is None else tuple(int(v) for v in shard)
+        if self.shard is not None:
+            self._h = lib().det_linear_plan_shard(self.M, self.N, self.K, *self.shard, self.wfmt)
+        elif self.wfmt == DET_WEIGHT_BF16:
             self._h = lib().det_linear_plan(self.M, self.N, self.K)
         else:
             self._h = lib().det_linear_plan_w(self.M, self.N, self.K, self.wfmt)
@@ -164,6 +170,30 @@ def det_linear_plan(M: int, N: int, K: int) -> Plan:
 def det_linear_plan_w(M: int, N: int, K: int, wfmt) -> Plan:
     """Plan for weights stored as "bf16" / "fp16" / "fp32" (or the det_weight_format_t value)."""
     return Plan(M, N, K, wfmt)
+
+
+def det_linear_plan_shard(M: int, N: int, K: int, n_begin: int, n_count: int, ldy: int, wfmt="bf16") -> Plan:
+    """Plan for the column shard [n_begin, n_begin + n_count) of the layer (M, N, K); the order is the
+    whole layer's, so the shard's outputs have the bits of the same columns of det_linear_plan(M, N, K)."""
+    return Plan(M, N, K, wfmt, shard=(n_begin, n_count, ldy))
+
+
+def det_linear_run_shard(plan: Plan, x, W_shard, b_shard, y_cols, stream=None) -> None:
+    """Run a shard plan.  W_shard [n_count, K] (the shard's weight rows), b_shard [n_count] or None,
+    y_cols: a [M, n_count] float32 CUDA view whose row stride is the plan's ldy and column stride 1
+    (e.g. y_full[:, n_begin:n_begin + n_count] for ldy = N)."""
+    n_begin, n_count, ldy = plan.shard
+    _expect(x, torch.float32, (plan.M, plan.K), "x")
+    _expect(W_shard, plan.w_dtype, (n_count, plan.K), "W_shard")
+    if b_shard is not None:
+        _expect(b_shard, torch.float32, (n_count,), "b_shard")
+    if (not y_cols.is_cuda or y_cols.dtype != torch.float32 or tuple(y_cols.shape) != (plan.M, n_count)
+            or y_cols.stride(1) != 1 or (plan.M > 1 and y_cols.stride(0) != ldy)):
+        raise ValueError(f"y_cols: need a float32 CUDA view of shape {(plan.M, n_count)} with strides ({ldy}, 1), "
+                         f"got {tuple(y_cols.shape)} strides {y_cols.stride()}")
+    _check(lib().det_linear_run_w(plan.handle, x.data_ptr(), W_shard.data_ptr(),
+                                  b_shard.data_ptr() if b_shard is not None else None, y_cols.data_ptr(),
+                                  _stream_ptr(stream)))
 
 
 def det_linear_plan_destroy(plan: Plan) -> None:

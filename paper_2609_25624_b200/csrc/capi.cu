@@ -71,7 +71,8 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const vo
     a.x = x; a.W = W; a.b = b; a.y = y;
     a.wfmt = p.weight_format;
     a.partials = plan->partials;
-    a.M = p.M; a.N = p.N; a.K = p.K;
+    a.M = p.M; a.N = plan->n_count; a.K = p.K;            // the kernels see the shard; the order is the layer's
+    a.ldy = plan->ldy;
     a.seg_len = p.seg_len; a.S = p.S;
     a.stream = stream;
     a.status = plan->status;
@@ -87,7 +88,7 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const vo
     cudaError_t e = cudaSuccess;
     if (kernel == kKernelDecode) {
         DecodeConfig cfg;
-        if (!decode_config_for(p.M, p.N, p.K, p.weight_format, plan->variant, &cfg)) {
+        if (!decode_config_for(p.M, plan->n_count, p.K, p.S, p.weight_format, plan->variant, &cfg)) {
             set_error("run: no decode configuration for this shape/variant");
             return DET_ERR_INVALID_ARG;
         }
@@ -95,7 +96,7 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const vo
             const CUtensorMapDataType wdt = p.weight_format == DET_WEIGHT_FP32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                             : p.weight_format == DET_WEIGHT_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
                                                                                  : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-            if (!encode_2d(&plan->map_w, wdt, p.weight_format == DET_WEIGHT_FP32 ? 4 : 2, W, (uint64_t)p.N, (uint64_t)p.K,
+            if (!encode_2d(&plan->map_w, wdt, p.weight_format == DET_WEIGHT_FP32 ? 4 : 2, W, (uint64_t)plan->n_count, (uint64_t)p.K,
                            (uint32_t)cfg.rt, (uint32_t)cfg.kc, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
                 return DET_ERR_CUDA;
             if (!encode_2d(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, x, (uint64_t)p.M, (uint64_t)p.K,
@@ -128,9 +129,21 @@ det_linear_plan_t* det_linear_plan(int64_t M, int64_t N, int64_t K) { return det
 
 det_linear_plan_t* det_linear_plan_w(int64_t M, int64_t N, int64_t K, int32_t wfmt)
 {
+    return det_linear_plan_shard(M, N, K, 0, N, N, wfmt);
+}
+
+det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K, int64_t n_begin, int64_t n_count, int64_t ldy,
+                                         int32_t wfmt)
+{
     det_linear_params_t prm;
     if (fill_params(M, N, K, &prm) != DET_OK) return nullptr;
     if (wfmt < DET_WEIGHT_BF16 || wfmt > DET_WEIGHT_FP32) { set_error("plan: unknown weight format %d", wfmt); return nullptr; }
+    if (n_begin < 0 || n_count < 1 || n_begin > N - n_count || ldy < n_count) {
+        set_error("plan: shard [%lld, %lld) with row pitch %lld does not fit a layer with N = %lld", (long long)n_begin,
+                  (long long)(n_begin + n_count), (long long)ldy, (long long)N);
+        return nullptr;
+    }
+    prm.workspace_bytes = prm.S > 1 ? 4ull * (uint64_t)prm.S * (uint64_t)M * (uint64_t)n_count : 0;
     prm.weight_format = wfmt;
     if (wfmt == DET_WEIGHT_FP32) prm.kernel = (K % 4 == 0) ? (prm.bucket == 0 ? kKernelDecode : kKernelPrefill) : kKernelGeneric;
     int dev = 0;
@@ -148,6 +161,9 @@ det_linear_plan_t* det_linear_plan_w(int64_t M, int64_t N, int64_t K, int32_t wf
     if (!plan) { set_error("plan: host allocation failed"); return nullptr; }
     memset(plan, 0, sizeof *plan);
     plan->prm = prm;
+    plan->n_begin = n_begin;
+    plan->n_count = n_count;
+    plan->ldy = ldy;
     plan->device = dev;
     plan->sm_count = prop.multiProcessorCount;
     plan->forced_kernel = -1;
@@ -191,6 +207,10 @@ static det_status_t run_host_impl(det_linear_plan_t* plan, const float* x_host, 
         return DET_ERR_INVALID_ARG;
     }
     const det_linear_params_t& p = plan->prm;
+    if (plan->n_count != p.N || plan->ldy != p.N) {
+        set_error("run_host: the plan is a column shard; use det_linear_run_w with device buffers");
+        return DET_ERR_INVALID_ARG;
+    }
     const size_t xb = (size_t)p.M * p.K * 4, yb = (size_t)p.M * p.N * 4;
     cudaError_t e;
     if (!plan->x_stage) {
@@ -255,7 +275,7 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
     char tiling[128] = "null";
     if (p.kernel == kKernelDecode) {
         DecodeConfig c;
-        if (decode_config_for(p.M, p.N, p.K, p.weight_format, plan->variant, &c))
+        if (decode_config_for(p.M, plan->n_count, p.K, p.S, p.weight_format, plan->variant, &c))
             snprintf(tiling, sizeof tiling, "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"kc\": %d, \"stages\": %d}", c.mt,
                      c.wm, c.rt, c.wr, c.kc, c.stages);
     }
@@ -267,10 +287,12 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
     int w = snprintf(buf, n,
                      "{\"M\": %lld, \"N\": %lld, \"K\": %lld, \"bucket\": \"%s\", \"V\": %d, \"L\": %d, \"P\": %d, "
                      "\"seg_len\": %lld, \"S\": %d, \"order_version\": %d, \"kernel\": \"%s\", \"workspace_bytes\": %llu, "
-                     "\"weight_format\": \"%s\", \"decode_tiling\": %s, \"prefill_tile\": %s}",
+                     "\"weight_format\": \"%s\", \"decode_tiling\": %s, \"prefill_tile\": %s, "
+                     "\"shard\": {\"n_begin\": %lld, \"n_count\": %lld, \"ldy\": %lld}}",
                      (long long)p.M, (long long)p.N, (long long)p.K, p.bucket == 0 ? "decode" : "prefill", p.V, p.L, p.P,
                      (long long)p.seg_len, p.S, p.order_version, kn[p.kernel], (unsigned long long)p.workspace_bytes,
-                     p.weight_format == DET_WEIGHT_FP32 ? "fp32" : p.weight_format == DET_WEIGHT_FP16 ? "fp16" : "bf16", tiling, ptile);
+                     p.weight_format == DET_WEIGHT_FP32 ? "fp32" : p.weight_format == DET_WEIGHT_FP16 ? "fp16" : "bf16", tiling, ptile,
+                     (long long)plan->n_begin, (long long)plan->n_count, (long long)plan->ldy);
     if (w < 0 || (size_t)w >= n) { set_error("describe: buffer too small (%d bytes needed)", w + 1); return DET_ERR_INVALID_ARG; }
     return DET_OK;
 }
@@ -325,7 +347,7 @@ det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
     if (!plan || variant < 0) { set_error("set_variant: bad argument"); return DET_ERR_INVALID_ARG; }
     if (plan->prm.bucket == 0) {
         DecodeConfig cfg;
-        if (!decode_config_for(plan->prm.M, plan->prm.N, plan->prm.K, plan->prm.weight_format, variant, &cfg)) {
+        if (!decode_config_for(plan->prm.M, plan->n_count, plan->prm.K, plan->prm.S, plan->prm.weight_format, variant, &cfg)) {
             set_error("set_variant: the decode kernel has fewer than %d tilings for this batch size", variant);
             return DET_ERR_INVALID_ARG;
         }

@@ -243,7 +243,7 @@ template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG, int WF>
 __global__ void __launch_bounds__((WM * WR + PG) * 32, (Cfg<MT, WM, RT, WR, KC, STAGES, PG, WF>::kMinBlocks))
 decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
               const float* __restrict__ bias, float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct,
-              int n_row_tiles, int n_mblocks, DeviceStatus* status)
+              int n_row_tiles, int n_mblocks, long long ldy, DeviceStatus* status)
 {
     using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG, WF>;
     extern __shared__ unsigned char smem_raw[];
@@ -446,7 +446,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                         float r0 = v[t];
                         if (direct) {
                             if (bias) r0 = __fadd_rn(r0, bv[t]);
-                            out[(long long)m * N + n] = r0;
+                            out[(long long)m * ldy + n] = r0;
                         } else {
                             out[((long long)un.s * M + m) * N + n] = r0;
                         }
@@ -507,7 +507,7 @@ cudaError_t launch_decode_t(const LaunchArgs& a, const CUtensorMap* map_w, const
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, *map_w, *map_x, a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N,
-                                       (int)a.K, (int)a.seg_len, a.S, direct, n_row_tiles, n_mblocks, a.status);
+                                       (int)a.K, (int)a.seg_len, a.S, direct, n_row_tiles, n_mblocks, (long long)a.ldy, a.status);
     if (e != cudaSuccess) return e;
     if (!direct) return launch_combine(a);
     return cudaSuccess;

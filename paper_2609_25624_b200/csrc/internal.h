@@ -29,7 +29,8 @@ struct LaunchArgs {
     const void* W;        // [N,K] in weight format wfmt
     int wfmt;             // det_weight_format_t
     const float* b;
-    float* y;             // final output [M,N]
+    float* y;             // final output [M,N], row pitch ldy
+    int64_t ldy;          // floats between consecutive rows of y (N unless the plan is a column shard)
     float* partials;      // [S,M,N] when S > 1, else nullptr
     int64_t M, N, K;
     int64_t seg_len;
@@ -56,7 +57,8 @@ struct DecodeConfig {
     int mt, wm, rt, wr, kc, stages;   // warp tile (mt x rt), warps (wm x wr), k per stage, ring depth
     int id;
 };
-bool decode_config_for(int64_t M, int64_t N, int64_t K, int wfmt, int variant, DecodeConfig* out);
+// S = number of K segments of the order (it only scales the unit count in the schedule's cost model)
+bool decode_config_for(int64_t M, int64_t N, int64_t K, int S, int wfmt, int variant, DecodeConfig* out);
 int decode_num_variants();
 
 }  // namespace detlin
@@ -65,7 +67,8 @@ struct det_linear_plan {
     det_linear_params_t prm;
     int device;
     int sm_count;
-    float* partials;                 // device, S*M*N floats or nullptr
+    float* partials;                 // device, S*M*n_count floats or nullptr
+    int64_t n_begin, n_count, ldy;   // column shard computed by this plan (0, N, N for a whole layer)
     detlin::DeviceStatus* status;    // device
     float* x_stage;                  // device staging for det_linear_run_host
     float* y_stage;

@@ -66,8 +66,9 @@ int decode_num_variants()
 
 // variant 0 = automatic; variant v >= 1 = the v-th candidate tiling for this batch size (own class
 // first, then the 8-row tilings when M > 8).
-bool decode_config_for(int64_t M, int64_t N, int64_t K, int wfmt, int variant, DecodeConfig* out)
+bool decode_config_for(int64_t M, int64_t N, int64_t K, int S, int wfmt, int variant, DecodeConfig* out)
 {
+    (void)K;
     int classes[2];
     const int n_classes = candidate_classes(M, classes);
     int total = 0;
@@ -79,9 +80,6 @@ bool decode_config_for(int64_t M, int64_t N, int64_t K, int wfmt, int variant, D
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             sms = 148;
-        // the split factor does not depend on the tiling; recompute it from the shape
-        det_linear_params_t prm;
-        const int S = fill_params(M, N, K, &prm) == DET_OK ? prm.S : 1;
         double best = 1e301;
         for (int ci = 0; ci < n_classes; ++ci) {
             const DecodeClassTable* t = class_table(wfmt, classes[ci]);
@@ -106,7 +104,7 @@ bool decode_config_for(int64_t M, int64_t N, int64_t K, int wfmt, int variant, D
 cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
 {
     DecodeConfig cfg;
-    if (!decode_config_for(a.M, a.N, a.K, a.wfmt, a.variant, &cfg)) return cudaErrorInvalidValue;
+    if (!decode_config_for(a.M, a.N, a.K, a.S, a.wfmt, a.variant, &cfg)) return cudaErrorInvalidValue;
     return class_table(a.wfmt, cfg.id / 64)->entries[cfg.id % 64].fn(a, map_w, map_x);
 }
 

@@ -13,7 +13,7 @@ namespace detlin {
 template <int WF>
 __global__ void __launch_bounds__(256)
 generic_decode_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type* __restrict__ W, const float* __restrict__ b,
-                      float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct)
+                      float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct, int64_t ldy)
 {
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -36,7 +36,7 @@ generic_decode_kernel(const float* __restrict__ x, const typename WeightElem<WF>
         }
         const float t = lane_tree_sum(a);
         if (lane == 0) {
-            if (direct) out[m * N + n] = b ? __fadd_rn(t, b[n]) : t;
+            if (direct) out[m * ldy + n] = b ? __fadd_rn(t, b[n]) : t;
             else        out[((int64_t)s * M + m) * N + n] = t;
         }
     }
@@ -46,7 +46,7 @@ generic_decode_kernel(const float* __restrict__ x, const typename WeightElem<WF>
 template <int WF>
 __global__ void __launch_bounds__(256)
 generic_prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type* __restrict__ W, const float* __restrict__ b,
-                       float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct)
+                       float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct, int64_t ldy)
 {
     const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t m = blockIdx.y;
@@ -58,7 +58,7 @@ generic_prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF
     const typename WeightElem<WF>::type* wrow = W + n * K;
     float t = 0.0f;
     for (int64_t k = k_lo; k < k_hi; ++k) t = __fmaf_rn(xrow[k], up_elem<WF>(wrow[k]), t);
-    if (direct) out[m * N + n] = b ? __fadd_rn(t, b[n]) : t;
+    if (direct) out[m * ldy + n] = b ? __fadd_rn(t, b[n]) : t;
     else        out[((int64_t)s * M + m) * N + n] = t;
 }
 
@@ -66,13 +66,14 @@ generic_prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF
 // order by one thread, then the bias; no atomics anywhere.
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ partials, const float* __restrict__ b, float* __restrict__ y,
-               int64_t MN, int64_t N, int S)
+               int64_t MN, int64_t N, int S, int64_t ldy)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= MN) return;
     float t = partials[i];
     for (int s = 1; s < S; ++s) t = __fadd_rn(t, partials[(int64_t)s * MN + i]);
-    y[i] = b ? __fadd_rn(t, b[i % N]) : t;
+    const int64_t m = i / N, n = i % N;
+    y[m * ldy + n] = b ? __fadd_rn(t, b[n]) : t;
 }
 
 template <int WF>
@@ -85,15 +86,15 @@ static cudaError_t launch_generic_t(const LaunchArgs& a, int bucket)
     if (bucket == 0) {
         const int64_t warps = a.N * a.S;
         const int64_t blocks = (warps + 7) / 8;
-        generic_decode_kernel<WF><<<(unsigned)blocks, 256, 0, a.stream>>>(a.x, W, a.b, out, a.M, a.N, a.K, a.seg_len, a.S, direct);
+        generic_decode_kernel<WF><<<(unsigned)blocks, 256, 0, a.stream>>>(a.x, W, a.b, out, a.M, a.N, a.K, a.seg_len, a.S, direct, a.ldy);
     } else {
         // grid.y carries M (< 65536 per launch); larger M is cut into slabs of rows
         const int64_t max_y = 32768;
         for (int64_t m0 = 0; m0 < a.M; m0 += max_y) {
             const int64_t mm = (a.M - m0 < max_y) ? a.M - m0 : max_y;
             dim3 grid((unsigned)((a.N + 255) / 256), (unsigned)mm, (unsigned)a.S);
-            float* o = out + m0 * a.N;   // both layouts ([M][N] and [s][M][N]) advance by whole rows
-            generic_prefill_kernel<WF><<<grid, 256, 0, a.stream>>>(a.x + m0 * a.K, W, a.b, o, a.M, a.N, a.K, a.seg_len, a.S, direct);
+            float* o = out + m0 * (direct ? a.ldy : a.N);   // both layouts ([M][ldy] and [s][M][N]) advance by whole rows
+            generic_prefill_kernel<WF><<<grid, 256, 0, a.stream>>>(a.x + m0 * a.K, W, a.b, o, a.M, a.N, a.K, a.seg_len, a.S, direct, a.ldy);
         }
     }
     cudaError_t e = cudaGetLastError();
@@ -112,7 +113,7 @@ cudaError_t launch_generic(const LaunchArgs& a, int bucket)
 cudaError_t launch_combine(const LaunchArgs& a)
 {
     const int64_t MN = a.M * a.N;
-    combine_kernel<<<(unsigned)((MN + 255) / 256), 256, 0, a.stream>>>(a.partials, a.b, a.y, MN, a.N, a.S);
+    combine_kernel<<<(unsigned)((MN + 255) / 256), 256, 0, a.stream>>>(a.partials, a.b, a.y, MN, a.N, a.S, a.ldy);
     return cudaGetLastError();
 }
 

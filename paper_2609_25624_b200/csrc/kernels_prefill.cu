@@ -68,7 +68,8 @@ __device__ __forceinline__ void lds_floats(uint32_t addr, float* v)
 template <int WF, int TR>
 __global__ void __launch_bounds__(kThreads, 2)
 prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type* __restrict__ W, const float* __restrict__ bias,
-               float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct, int tiles_m, int tiles_n)
+               float* __restrict__ out, int M, int N, int K, int seg_len, int S, int direct, int tiles_m, int tiles_n,
+               long long ldy)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t smem = (uint32_t)__cvta_generic_to_shared(smem_raw);
@@ -223,12 +224,12 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
     }
 
     // ---- epilogue: bias (direct) or the segment's partial ----
-    const bool vec_ok = (N % 4 == 0);
+    const bool vec_ok = direct ? (ldy % 4 == 0) : (N % 4 == 0);     // rows of the destination start 16-byte aligned
 #pragma unroll
     for (int i = 0; i < TR; ++i) {
         const int m = m0 + (i < 4 ? 4 * ty + i : 64 + TB * ty + (i - 4));
         if (m >= M) continue;
-        float* orow = direct ? out + (long long)m * N : out + ((long long)s * M + m) * N;
+        float* orow = direct ? out + (long long)m * ldy : out + ((long long)s * M + m) * N;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int n = n0 + 64 * h + 4 * tx;
@@ -269,7 +270,7 @@ cudaError_t launch_prefill_t(const LaunchArgs& a)
     const int direct = (a.S == 1);
     prefill_kernel<WF, TR><<<(unsigned)units, kThreads, kSmemBytes, a.stream>>>(
         a.x, static_cast<const typename WeightElem<WF>::type*>(a.W), a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N,
-        (int)a.K, (int)a.seg_len, a.S, direct, tiles_m, tiles_n);
+        (int)a.K, (int)a.seg_len, a.S, direct, tiles_m, tiles_n, (long long)a.ldy);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (!direct) return launch_combine(a);

@@ -70,7 +70,7 @@ extern "C" det_status_t det_linear_run_noalloc(int64_t M, int64_t N, int64_t K, 
     a.x = x; a.W = W; a.b = b; a.y = y;
     a.wfmt = DET_WEIGHT_BF16;
     a.partials = p.S > 1 ? scratch : nullptr;    // every partial is written by the first pass before the
-    a.M = M; a.N = N; a.K = K;                   // second pass reads it: nothing has to start at zero
+    a.M = M; a.N = N; a.K = K; a.ldy = N;                   // second pass reads it: nothing has to start at zero
     a.seg_len = p.seg_len; a.S = p.S;
     a.stream = static_cast<cudaStream_t>(stream);
     e = launch_generic(a, p.bucket);
