@@ -318,6 +318,7 @@ def run_own(args, world, rank, local):
         line["layercast_style_reference"] = layercast_table(work, st, line["per_case"])
         line["weight_formats"] = weight_format_table(B, dev, st, hbm_peak, fp32_peak)
         line["column_shards"] = shard_table(B, dev, st, hbm_peak)
+        line["r3_ablation"] = ablation_table(B, dev, st)
         line["cpu_baseline"] = cpu_baseline(work)
         for w in work:                       # free the sweep's 2.2 GB before the 15 GB stack
             w["plan"].close()
@@ -330,6 +331,11 @@ def run_own(args, world, rank, local):
     # traffic is proportional to the algorithmic bytes, so it is scaled to the step's average launch here.
     line["roofline"]["traffic"] = DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes / launches_per_step
     line["roofline"]["algorithmic_bytes_per_launch"] = alg_bytes / launches_per_step
+    # Each launch against the roof that binds IT: max(bytes / HBM peak, flops / FP32 CUDA-core peak).
+    t_bind = sum(max(algorithmic_bytes(M, N, K) / (hbm_peak * 1e9), 2.0 * M * N * K / (fp32_peak * 1e12))
+                 for (M, N, K, _) in decode_cases())
+    line["roofline"]["binding_roof_ms_per_step"] = t_bind * 1e3
+    line["roofline"]["frac_of_binding_roof"] = t_bind * 1e3 / ms_step
     print(json.dumps(line), flush=True)
     for w in work:
         w["plan"].close()
@@ -484,6 +490,31 @@ def shard_table(B, dev, st, hbm_peak):
                              "weight_gbs_per_rank": wbytes / ms / 1e6, "pct_hbm": 100 * wbytes / ms / 1e6 / hbm_peak})
             del Ws
     return rows
+
+
+def ablation_table(B, dev, st):
+    """Rule R3 ablation (supplement C of the paper): distinct outputs in 50 runs and time per call of the
+    library's ordered split-K against a test-only atomicAdd combine of the same partials."""
+    import hashlib
+    M, N, K = 8, 512, 4096
+    x, W, b = inputs.make_case(M, N, K)
+    xd, Wd, bd = x.to(dev), W.to(dev), b.to(dev)
+    y = torch.empty(M, N, dtype=torch.float32, device=dev)
+    plan = B.det_linear_plan(M, N, K)
+    S = B.det_linear_plan_get_params(plan).S
+    digests = {"ordered": set(), "atomic": set()}
+    with torch.cuda.stream(st):
+        for _ in range(50):
+            B.det_linear_run(plan, xd, Wd, bd, y)
+            digests["ordered"].add(hashlib.sha256(y.cpu().numpy().tobytes()).hexdigest())
+            B.det_test_linear_atomic_splitk(xd, Wd, bd, y, S)
+            digests["atomic"].add(hashlib.sha256(y.cpu().numpy().tobytes()).hexdigest())
+    us_ordered = time_graph(lambda: [B.det_linear_run(plan, xd, Wd, bd, y) for _ in range(16)], 3, st) / 16 * 1e3
+    us_atomic = time_graph(lambda: [B.det_test_linear_atomic_splitk(xd, Wd, bd, y, S) for _ in range(16)], 3, st) / 16 * 1e3
+    plan.close()
+    return {"shape": [M, N, K], "S": S, "runs": 50, "distinct_ordered": len(digests["ordered"]),
+            "distinct_atomic": len(digests["atomic"]), "us_ordered": us_ordered, "us_atomic_control": us_atomic,
+            "note": "the atomic control is an untuned one-warp-per-row kernel; its time is context, not a comparison"}
 
 
 def lm_head_table(B, dev, st, hbm_peak, fp32_peak):

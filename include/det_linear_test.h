@@ -49,6 +49,17 @@ DET_API void det_test_green_stream_destroy(void* handle);
 DET_API det_status_t det_test_measure_fma_peak(int packed, double* tflops_out);
 DET_API det_status_t det_test_measure_read_bandwidth(const void* buf, size_t bytes, double* gbs_out);
 
+/*
+ * Negative control for rule R3 (the paper's split-K ablation "none / ordered / atomic"): the decode
+ * order's segment partials for a requested split S_req (segments of whole 256-element blocks, as in
+ * the library), combined with atomicAdd onto y (pre-set to the bias, or zero) in arrival order --
+ * the scheme the rule forbids.  The output is close to det_linear_run's but its bits depend on grid
+ * scheduling and may change from run to run.  BF16 weights, device pointers, layouts as for
+ * det_linear_run; enqueued on `stream`.  Nothing in the library uses it.
+ */
+DET_API det_status_t det_test_linear_atomic_splitk(int64_t M, int64_t N, int64_t K, int32_t S_req, const float* x,
+                                                   const uint16_t* W, const float* b, float* y, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

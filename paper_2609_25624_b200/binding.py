@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.det_test_green_stream_destroy.restype = None
         L.det_linear_run_noalloc.argtypes = [i64, i64, i64, p, p, p, p, p]
         L.det_linear_run_noalloc.restype = i32
+        L.det_test_linear_atomic_splitk.argtypes = [i64, i64, i64, ctypes.c_int32, p, p, p, p, p]
+        L.det_test_linear_atomic_splitk.restype = i32
         L.det_test_measure_fma_peak.argtypes = [i32, ctypes.POINTER(ctypes.c_double)]
         L.det_test_measure_fma_peak.restype = i32
         L.det_test_measure_read_bandwidth.argtypes = [p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_double)]
@@ -322,3 +324,16 @@ def det_test_measure_read_bandwidth(buf) -> float:
     out = ctypes.c_double(0.0)
     _check(lib().det_test_measure_read_bandwidth(buf.data_ptr(), buf.numel() * buf.element_size(), ctypes.byref(out)))
     return out.value
+
+
+def det_test_linear_atomic_splitk(x, W, b, y, S_req: int, stream=None) -> None:
+    """Negative control for rule R3: split-K partials combined with atomicAdd in arrival order."""
+    M, K = x.shape
+    N = W.shape[0]
+    _expect(x, torch.float32, (M, K), "x")
+    _expect(W, torch.bfloat16, (N, K), "W")
+    _expect(y, torch.float32, (M, N), "y")
+    if b is not None:
+        _expect(b, torch.float32, (N,), "b")
+    _check(lib().det_test_linear_atomic_splitk(M, N, K, int(S_req), x.data_ptr(), W.data_ptr(),
+                                               b.data_ptr() if b is not None else None, y.data_ptr(), _stream_ptr(stream)))
