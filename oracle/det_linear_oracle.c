@@ -245,6 +245,54 @@ int det_oracle_argmax_rows(const float *y, int64_t M, int64_t N, int32_t *idx)
     return 0;
 }
 
+/* ---- fixed-order RMSNorm ---------------------------------------------------------------------
+ * An extension in the paper's spirit, not one of its kernels: the paper leaves RMSNorm to vendor
+ * FP32 kernels and names the reductions outside the linear layers as the residual channel of
+ * divergence.  Here the row's sum of squares is reduced in the decode order family
+ * (V = 4, L = 32, P = 1, one segment): chunks of 128 elements ascending, lane l owns the 4
+ * consecutive elements c + 4 l + j, each element enters its lane's accumulator with one
+ * fmaf(x, x, acc) from +0.0f, elements beyond H are skipped, and the 32 lane sums are added by the
+ * balanced tree, adjacent lanes first.  Then, each step one IEEE binary32 operation:
+ *     mean = ss / (float)H;  t = mean + eps;  r = 1.0f / sqrtf(t);  y[h] = (x[h] * r) * g[h].
+ */
+float det_oracle_sum_squares(const float *x, int64_t H)
+{
+    unsigned mx = oracle_enter_ieee();
+    float a[32];
+    for (int l = 0; l < 32; ++l) a[l] = 0.0f;
+    for (int64_t c = 0; c < H; c += 128)
+        for (int l = 0; l < 32; ++l)
+            for (int j = 0; j < 4; ++j) {
+                const int64_t k = c + 4 * (int64_t)l + j;
+                if (k < H) a[l] = fmaf(x[k], x[k], a[l]);
+            }
+    for (int w = 32; w > 1; w /= 2)
+        for (int i = 0; i < w / 2; ++i) a[i] = a[2 * i] + a[2 * i + 1];
+    oracle_leave_ieee(mx);
+    return a[0];
+}
+
+int det_oracle_rmsnorm(const float *x, const float *g, float eps, int64_t M, int64_t H, float *y)
+{
+    if (M < 0 || H < 1 || !x || !g || !y) return 1;
+    unsigned mx = oracle_enter_ieee();
+    for (int64_t m = 0; m < M; ++m) {
+        const float *xr = x + m * H;
+        float *yr = y + m * H;
+        const float ss = det_oracle_sum_squares(xr, H);
+        const float mean = ss / (float)H;
+        const float t = mean + eps;
+        const float root = sqrtf(t);
+        const float r = 1.0f / root;
+        for (int64_t h = 0; h < H; ++h) {
+            const float xs = xr[h] * r;
+            yr[h] = xs * g[h];
+        }
+    }
+    oracle_leave_ieee(mx);
+    return 0;
+}
+
 int det_oracle_threads(void)
 {
 #ifdef _OPENMP

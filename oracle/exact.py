@@ -123,3 +123,65 @@ def linear(x, W_bits, b, V, L, P, seg_len, wfmt="bf16"):
     return [[output(list(map(float, xr)), list(map(conv, wr)), None if b is None else float(b[n]),
                     V, L, P, seg_len, wfmt)
              for n, wr in enumerate(W_bits)] for xr in x]
+
+
+# ---- fixed-order RMSNorm, exact-rational version --------------------------------------------------
+
+def mul32(a: float, b: float) -> float:
+    """binary32 multiplication, one rounding (finite, nonzero-sign handling as for add32)."""
+    q = Fraction(a) * Fraction(b)
+    if q == 0:
+        return -0.0 if (_is_neg(a) != _is_neg(b)) else 0.0
+    return round_to_binary32(q)
+
+
+def div32(a: float, b: float) -> float:
+    """binary32 division a / b, one rounding; b != 0."""
+    q = Fraction(a) / Fraction(b)
+    if q == 0:
+        return -0.0 if (_is_neg(a) != _is_neg(b)) else 0.0
+    return round_to_binary32(q)
+
+
+def sqrt32(t: float) -> float:
+    """Correctly rounded binary32 square root of t >= 0.  The root is bracketed to 2^-160 with an
+    integer square root; a binary32 rounding boundary (a 25-bit number) can only be hit exactly by
+    a perfect square, which is detected, so a point strictly inside the bracket rounds correctly."""
+    if t == 0:
+        return t
+    q = Fraction(t)
+    k = 160
+    scaled = q * Fraction(4) ** k                    # t * 2^(2k)
+    num = scaled.numerator // scaled.denominator
+    exact_int = scaled.denominator == 1
+    n = math.isqrt(num)
+    if exact_int and n * n == num:
+        return round_to_binary32(Fraction(n, 2 ** k))
+    return round_to_binary32(Fraction(2 * n + 1, 2 ** (k + 1)))
+
+
+def sum_squares(xrow) -> float:
+    """Decode-order sum of squares: chunks of 128 ascending, lane l owns 4 consecutive elements,
+    fma(x, x, acc) from +0, tails skipped, adjacent-first tree over the 32 lanes."""
+    H = len(xrow)
+    lanes = [0.0] * 32
+    for c in range(0, H, 128):
+        for l in range(32):
+            for j in range(4):
+                k = c + 4 * l + j
+                if k < H:
+                    lanes[l] = fma32(xrow[k], xrow[k], lanes[l])
+    w = 32
+    while w > 1:
+        lanes = [add32(lanes[2 * i], lanes[2 * i + 1]) for i in range(w // 2)]
+        w //= 2
+    return lanes[0]
+
+
+def rmsnorm_row(xrow, g, eps: float):
+    H = len(xrow)
+    ss = sum_squares(xrow)
+    mean = div32(ss, round_to_binary32(Fraction(H)))
+    t = add32(mean, eps)
+    r = div32(1.0, sqrt32(t))
+    return [mul32(mul32(xv, r), gv) for xv, gv in zip(xrow, g)]

@@ -102,6 +102,10 @@ def lib() -> ctypes.CDLL:
         L.det_oracle_up.argtypes = [ctypes.c_uint16]
         L.det_oracle_up.restype = ctypes.c_float
         L.det_oracle_threads.restype = i32
+        L.det_oracle_sum_squares.argtypes = [p, i64]
+        L.det_oracle_sum_squares.restype = ctypes.c_float
+        L.det_oracle_rmsnorm.argtypes = [p, p, ctypes.c_float, i64, i64, p]
+        L.det_oracle_rmsnorm.restype = i32
         _lib = L
     return _lib
 
@@ -183,6 +187,25 @@ def argmax_rows(y):
     if rc != 0:
         raise ValueError("det_oracle_argmax_rows rejected its arguments")
     return idx
+
+
+def sum_squares(x) -> float:
+    """Fixed-order sum of squares of one row (the reduction inside rmsnorm)."""
+    x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
+    return float(lib().det_oracle_sum_squares(x.ctypes.data, x.size))
+
+
+def rmsnorm(x, g, eps: float):
+    """Fixed-order RMSNorm per row: y = (x * r) * g, r = 1 / sqrt(sum_squares(x) / H + eps), every
+    step one binary32 operation.  x [M,H] float32, g [H] float32."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    M, H = x.shape
+    g = _f32(g, (H,))
+    y = np.empty((M, H), dtype=np.float32)
+    rc = lib().det_oracle_rmsnorm(x.ctypes.data, g.ctypes.data, float(np.float32(eps)), M, H, y.ctypes.data)
+    if rc != 0:
+        raise ValueError("det_oracle_rmsnorm rejected its arguments")
+    return y
 
 
 def up(h: int) -> float:
