@@ -319,6 +319,7 @@ def run_own(args, world, rank, local):
         line["weight_formats"] = weight_format_table(B, dev, st, hbm_peak, fp32_peak)
         line["column_shards"] = shard_table(B, dev, st, hbm_peak)
         line["r3_ablation"] = ablation_table(B, dev, st)
+        line["rmsnorm"] = rmsnorm_table(B, dev, st, hbm_peak)
         line["cpu_baseline"] = cpu_baseline(work)
         for w in work:                       # free the sweep's 2.2 GB before the 15 GB stack
             w["plan"].close()
@@ -515,6 +516,26 @@ def ablation_table(B, dev, st):
     return {"shape": [M, N, K], "S": S, "runs": 50, "distinct_ordered": len(digests["ordered"]),
             "distinct_atomic": len(digests["atomic"]), "us_ordered": us_ordered, "us_atomic_control": us_atomic,
             "note": "the atomic control is an untuned one-warp-per-row kernel; its time is context, not a comparison"}
+
+
+def rmsnorm_table(B, dev, st, hbm_peak):
+    """Fixed-order RMSNorm, H = 4096 (the Llama-3-8B hidden size): decode batches (launch-bound) and
+    prefill-sized batches whose input + output exceed L2 (HBM-bound: 8 M H bytes per call)."""
+    H = 4096
+    rows = []
+    g = torch.ones(H, device=dev)
+    for M in (1, 32, 2048, 16384):
+        x = torch.randn(M, H, generator=torch.Generator().manual_seed(M)).to(dev)
+        y = torch.empty_like(x)
+        reps = 16 if M <= 2048 else 4
+        with torch.cuda.stream(st):
+            B.det_rmsnorm(x, g, 1e-5, y)
+            torch.cuda.synchronize()
+        ms = time_graph(lambda: [B.det_rmsnorm(x, g, 1e-5, y) for _ in range(reps)], 3, st) / reps
+        nbytes = 8 * M * H
+        rows.append({"M": M, "H": H, "us": ms * 1e3, "gbs": nbytes / ms / 1e6, "pct_hbm": 100 * nbytes / ms / 1e6 / hbm_peak,
+                     "l2_resident": nbytes < (100 << 20)})
+    return rows
 
 
 def lm_head_table(B, dev, st, hbm_peak, fp32_peak):

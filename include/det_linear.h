@@ -187,6 +187,22 @@ DET_API void det_linear_plan_destroy(det_linear_plan_t* plan);
 DET_API det_status_t det_argmax_rows(const float* y, int64_t M, int64_t N, int32_t* idx, void* stream);
 
 /*
+ * Fixed-order RMSNorm per row: y[m,h] = (x[m,h] * r[m]) * g[h] with r = 1 / sqrt(ss / H + eps).
+ * An extension, not one of the paper's kernels: the paper keeps vendor FP32 RMSNorm and names the
+ * reductions outside the linear layers as the residual channel of cross-run divergence.  The row's
+ * sum of squares ss is reduced in the decode order of this header (chunks of 128 ascending, lane l
+ * owns 4 consecutive elements, one fmaf(x, x, acc) per element from +0.0f, elements beyond H
+ * skipped, 32 lane sums added by the adjacent-first tree); then one IEEE binary32 operation per step:
+ * mean = ss / float(H), t = mean + eps, root = sqrt(t), r = 1 / root, y = (x * r) * g.  The bits do
+ * not depend on M, the grid, the stream or the SM count.
+ *   x : device FP32 [M,H] row-major;  g : device FP32 [H];  y : device FP32 [M,H], must not overlap x
+ *   eps >= 0;  1 <= M, H < 2^31.  16-byte aligned buffers with H % 4 == 0 take vector loads.
+ * Enqueued on `stream`, no synchronisation, no allocation.
+ */
+DET_API det_status_t det_rmsnorm(const float* x, const float* g, float eps, int64_t M, int64_t H, float* y,
+                                 void* stream);
+
+/*
  * The same computation for callers that cannot allocate (the paper has no counterpart for this
  * entry point).  A host that owns all device memory through its own pool or arena, a plugin that
  * may not allocate after initialisation, or a latency-critical loop that cannot afford the

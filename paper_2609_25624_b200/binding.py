@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.det_linear_plan_destroy.restype = None
         L.det_argmax_rows.argtypes = [p, i64, i64, p, p]
         L.det_argmax_rows.restype = i32
+        L.det_rmsnorm.argtypes = [p, p, ctypes.c_float, i64, i64, p, p]
+        L.det_rmsnorm.restype = i32
         L.det_last_error.restype = ctypes.c_char_p
         L.det_order_version.restype = i32
         L.det_test_plan_force_kernel.argtypes = [p, i32]
@@ -279,6 +281,15 @@ def det_linear_run_noalloc(x, W, b, y, stream=None) -> None:
 
 def det_linear_plan_check(plan: Plan, stream=None) -> None:
     _check(lib().det_linear_plan_check(plan.handle, _stream_ptr(stream)))
+
+
+def det_rmsnorm(x, g, eps: float, y, stream=None) -> None:
+    """Fixed-order RMSNorm of the rows of x [M,H] with gain g [H] into y [M,H] (a different buffer)."""
+    M, H = x.shape
+    _expect(x, torch.float32, (M, H), "x")
+    _expect(g, torch.float32, (H,), "g")
+    _expect(y, torch.float32, (M, H), "y")
+    _check(lib().det_rmsnorm(x.data_ptr(), g.data_ptr(), float(eps), M, H, y.data_ptr(), _stream_ptr(stream)))
 
 
 def det_argmax_rows(y, idx, stream=None) -> None:

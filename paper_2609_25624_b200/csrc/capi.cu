@@ -244,6 +244,24 @@ det_status_t det_linear_run_host_async(det_linear_plan_t* plan, const float* x_h
     return run_host_impl(plan, x_host, W, b, y_host, stream, false);
 }
 
+det_status_t det_rmsnorm(const float* x, const float* g, float eps, int64_t M, int64_t H, float* y, void* stream)
+{
+    if (!x || !g || !y || M < 1 || H < 1 || H >= (1ll << 31) || M >= (1ll << 31)) {
+        set_error("rmsnorm: NULL pointer or size out of range (1 <= M, H < 2^31)");
+        return DET_ERR_INVALID_ARG;
+    }
+    if (!(eps >= 0.0f)) { set_error("rmsnorm: eps must be a non-negative number"); return DET_ERR_INVALID_ARG; }
+    int dev = 0;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) return cuda_fail("rmsnorm: device query", e);
+    if (prop.major != 10) { set_error("rmsnorm: device %d is sm_%d%d; this library is built for sm_100a only", dev, prop.major, prop.minor); return DET_ERR_ARCH; }
+    e = launch_rmsnorm(x, g, eps, M, H, y, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail("rmsnorm: launch", e);
+    return DET_OK;
+}
+
 det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream)
 {
     if (!plan) { set_error("check: plan is NULL"); return DET_ERR_INVALID_ARG; }

@@ -49,6 +49,8 @@ cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const C
 cudaError_t launch_prefill(const LaunchArgs& a);
 // rows per thread (tile height = 16 x this) the prefill kernel uses for batch size M; schedule only
 int prefill_rows_per_thread(int64_t M);
+// Fixed-order RMSNorm of M rows of H elements (rmsnorm.cu).
+cudaError_t launch_rmsnorm(const float* x, const float* g, float eps, int64_t M, int64_t H, float* y, cudaStream_t stream);
 cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cudaStream_t stream);
 
 // Decode-kernel tiling chosen for a shape (numerically inert); used by the host to build the
