@@ -158,6 +158,22 @@ DET_API det_status_t det_linear_run_host_async(det_linear_plan_t* plan, const fl
                                        const float* b, float* y_host, void* stream);
 
 /*
+ * Optional: time the plan's candidate thread-block tilings on the caller's buffers and pin the
+ * fastest one in the plan.  Only the schedule is chosen: tile sizes, warp counts and ring depth
+ * do not enter the reduction order (supplement C on rule R2 calls them numerically inert), every
+ * candidate produces the same bits, and the order parameters (V, L, P, S) remain the pure function
+ * of the shape that rule R2 asks for -- this is not the numeric autotuning the rule forbids.
+ * Without this call a cost model picks the tiling from the shape and the SM count.
+ * Plans of the decode bucket only; for other plans the call does nothing and reports variant 0.
+ * Runs every candidate six times on `stream` (CUDA events; a 192 MiB scratch buffer, allocated
+ * and freed inside the call, is read through L2 before each timed run so that the weights come
+ * from HBM) and synchronises; y holds the layer's result afterwards.  Do not call during stream capture.
+ * *variant_out (may be NULL): the pinned candidate's number; *best_us_out (may be NULL): its time.
+ */
+DET_API det_status_t det_linear_plan_tune(det_linear_plan_t* plan, const float* x, const void* W, const float* b,
+                                          float* y, void* stream, int32_t* variant_out, float* best_us_out);
+
+/*
  * Synchronise `stream` and report whether any kernel launched through this plan gave up a bounded
  * device-side wait (every wait on a TMA completion barrier is limited; on expiry the kernel
  * records the fact and returns instead of spinning).  DET_OK, DET_ERR_DEVICE_TIMEOUT or
@@ -168,8 +184,9 @@ DET_API det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream
 /* Copy the plan's order parameters to *out. */
 DET_API det_status_t det_linear_plan_get_params(const det_linear_plan_t* plan, det_linear_params_t* out);
 
-/* Write a JSON description (bucket, V, L, P, S, seg_len, order_version, kernel, workspace_bytes and,
- * for the decode kernel, the tiling the scheduler would pick on the current device -- schedule only)
+/* Write a JSON description (bucket, V, L, P, S, seg_len, order_version, kernel, workspace_bytes, the shard
+ * and, for the decode kernel, the tiling in use on the current device with its resident blocks per SM --
+ * schedule only)
  * to buf (at most n bytes including the terminator).  DET_ERR_INVALID_ARG if it does not fit. */
 DET_API det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, size_t n);
 

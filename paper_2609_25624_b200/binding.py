@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.det_linear_run_host.restype = i32
         L.det_linear_run_host_async.argtypes = [p, p, p, p, p, p]
         L.det_linear_run_host_async.restype = i32
+        L.det_linear_plan_tune.argtypes = [p, p, p, p, p, p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_float)]
+        L.det_linear_plan_tune.restype = i32
         L.det_linear_plan_check.argtypes = [p, p]
         L.det_linear_plan_check.restype = i32
         L.det_linear_plan_get_params.argtypes = [p, ctypes.POINTER(Params)]
@@ -277,6 +279,21 @@ def det_linear_run_noalloc(x, W, b, y, stream=None) -> None:
         _expect(b, torch.float32, (N,), "b")
     _check(lib().det_linear_run_noalloc(M, N, K, x.data_ptr(), W.data_ptr(), b.data_ptr() if b is not None else None,
                                         y.data_ptr(), _stream_ptr(stream)))
+
+
+def det_linear_plan_tune(plan: Plan, x, W, b, y, stream=None):
+    """Time the plan's candidate tilings on these buffers and pin the fastest (schedule only: every
+    candidate gives the same bits).  Returns (variant, microseconds); (0, -1.0) when there is nothing
+    to choose.  Synchronises the stream."""
+    n_count = plan.N if plan.shard is None else plan.shard[1]
+    _expect(x, torch.float32, (plan.M, plan.K), "x")
+    _expect(W, plan.w_dtype, (n_count, plan.K), "W")
+    if b is not None:
+        _expect(b, torch.float32, (n_count,), "b")
+    variant, us = ctypes.c_int32(0), ctypes.c_float(0.0)
+    _check(lib().det_linear_plan_tune(plan.handle, x.data_ptr(), W.data_ptr(), b.data_ptr() if b is not None else None,
+                                      y.data_ptr(), _stream_ptr(stream), ctypes.byref(variant), ctypes.byref(us)))
+    return int(variant.value), float(us.value)
 
 
 def det_linear_plan_check(plan: Plan, stream=None) -> None:

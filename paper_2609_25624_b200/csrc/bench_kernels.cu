@@ -57,6 +57,14 @@ __global__ void __launch_bounds__(512) read_stream_kernel(const uint4* __restric
     if (acc == 0x12345678u) out[0] = acc;
 }
 
+// Stream `bytes` of device memory through L2 (read only, so nothing is left dirty): used to evict a
+// weight matrix before a timed run.
+cudaError_t launch_l2_evict(const void* buf, size_t bytes, unsigned* sink, int sm_count, cudaStream_t stream)
+{
+    read_stream_kernel<<<sm_count * 8, 512, 0, stream>>>(static_cast<const uint4*>(buf), bytes / 16, sink);
+    return cudaGetLastError();
+}
+
 }  // namespace detlin
 
 using namespace detlin;

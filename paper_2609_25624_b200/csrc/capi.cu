@@ -262,6 +262,61 @@ det_status_t det_rmsnorm(const float* x, const float* g, float eps, int64_t M, i
     return DET_OK;
 }
 
+det_status_t det_linear_plan_tune(det_linear_plan_t* plan, const float* x, const void* W, const float* b, float* y,
+                                  void* stream, int32_t* variant_out, float* best_us_out)
+{
+    if (!plan || !x || !W || !y) { set_error("tune: plan, x, W and y must not be NULL"); return DET_ERR_INVALID_ARG; }
+    if (variant_out) *variant_out = 0;
+    if (best_us_out) *best_us_out = -1.0f;
+    const det_linear_params_t& p = plan->prm;
+    const int kernel = plan->forced_kernel >= 0 ? plan->forced_kernel : p.kernel;
+    if (kernel != kKernelDecode) return DET_OK;                     // one schedule only: nothing to choose
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // cold weights: a buffer larger than L2 is rewritten before every timed run (skipped if it cannot be had)
+    const size_t flush_bytes = 192u << 20;
+    void* flush = nullptr;
+    if (cudaMalloc(&flush, flush_bytes + 256) != cudaSuccess) { flush = nullptr; cudaGetLastError(); }
+    else if (cudaMemsetAsync(flush, 0, flush_bytes + 256, st) != cudaSuccess) { cudaGetLastError(); }
+    unsigned* sink = flush ? reinterpret_cast<unsigned*>(static_cast<char*>(flush) + flush_bytes) : nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    const int saved = plan->variant;
+    det_status_t status = DET_OK;
+    int best_variant = 0;
+    float best_ms = 0.0f;
+    if (e != cudaSuccess) status = cuda_fail("tune: event creation", e);
+    for (int v = 1; status == DET_OK; ++v) {
+        DecodeConfig cfg;
+        if (!decode_config_for(p.M, plan->n_count, p.K, p.S, p.weight_format, v, &cfg)) break;
+        plan->variant = v;
+        status = run_device(plan, x, W, b, y, st);                  // loads the kernel, builds the tensor maps
+        float v_ms = 0.0f;
+        for (int rep = 0; rep < 5 && status == DET_OK; ++rep) {
+            if (flush) e = launch_l2_evict(flush, flush_bytes, sink, plan->sm_count, st);
+            if (e == cudaSuccess) e = cudaEventRecord(e0, st);
+            if (e != cudaSuccess) { status = cuda_fail("tune: timing", e); break; }
+            status = run_device(plan, x, W, b, y, st);
+            if (status != DET_OK) break;
+            e = cudaEventRecord(e1, st);
+            if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+            float ms = 0.0f;
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+            if (e != cudaSuccess) { status = cuda_fail("tune: timing", e); break; }
+            if (rep == 0 || ms < v_ms) v_ms = ms;
+        }
+        if (status == DET_OK && (best_variant == 0 || v_ms < best_ms)) { best_variant = v; best_ms = v_ms; }
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (flush) cudaFree(flush);
+    if (status != DET_OK || best_variant == 0) { plan->variant = saved; return status; }
+    plan->variant = best_variant;
+    if (variant_out) *variant_out = best_variant;
+    if (best_us_out) *best_us_out = best_ms * 1e3f;
+    return DET_OK;
+}
+
 det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream)
 {
     if (!plan) { set_error("check: plan is NULL"); return DET_ERR_INVALID_ARG; }
@@ -290,12 +345,13 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
     if (!plan || !buf || n == 0) { set_error("describe: NULL argument"); return DET_ERR_INVALID_ARG; }
     const det_linear_params_t& p = plan->prm;
     static const char* kn[] = {"generic", "decode", "prefill"};
-    char tiling[128] = "null";
+    char tiling[160] = "null";
     if (p.kernel == kKernelDecode) {
         DecodeConfig c;
         if (decode_config_for(p.M, plan->n_count, p.K, p.S, p.weight_format, plan->variant, &c))
-            snprintf(tiling, sizeof tiling, "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"kc\": %d, \"stages\": %d}", c.mt,
-                     c.wm, c.rt, c.wr, c.kc, c.stages);
+            snprintf(tiling, sizeof tiling,
+                     "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"kc\": %d, \"stages\": %d, \"blocks_per_sm\": %d}", c.mt,
+                     c.wm, c.rt, c.wr, c.kc, c.stages, decode_config_occupancy(p.weight_format, c));
     }
     char ptile[64] = "null";
     if (p.kernel == kKernelPrefill) {
@@ -305,11 +361,11 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
     int w = snprintf(buf, n,
                      "{\"M\": %lld, \"N\": %lld, \"K\": %lld, \"bucket\": \"%s\", \"V\": %d, \"L\": %d, \"P\": %d, "
                      "\"seg_len\": %lld, \"S\": %d, \"order_version\": %d, \"kernel\": \"%s\", \"workspace_bytes\": %llu, "
-                     "\"weight_format\": \"%s\", \"decode_tiling\": %s, \"prefill_tile\": %s, "
+                     "\"weight_format\": \"%s\", \"variant\": %d, \"decode_tiling\": %s, \"prefill_tile\": %s, "
                      "\"shard\": {\"n_begin\": %lld, \"n_count\": %lld, \"ldy\": %lld}}",
                      (long long)p.M, (long long)p.N, (long long)p.K, p.bucket == 0 ? "decode" : "prefill", p.V, p.L, p.P,
                      (long long)p.seg_len, p.S, p.order_version, kn[p.kernel], (unsigned long long)p.workspace_bytes,
-                     p.weight_format == DET_WEIGHT_FP32 ? "fp32" : p.weight_format == DET_WEIGHT_FP16 ? "fp16" : "bf16", tiling, ptile,
+                     p.weight_format == DET_WEIGHT_FP32 ? "fp32" : p.weight_format == DET_WEIGHT_FP16 ? "fp16" : "bf16", plan->variant, tiling, ptile,
                      (long long)plan->n_begin, (long long)plan->n_count, (long long)plan->ldy);
     if (w < 0 || (size_t)w >= n) { set_error("describe: buffer too small (%d bytes needed)", w + 1); return DET_ERR_INVALID_ARG; }
     return DET_OK;

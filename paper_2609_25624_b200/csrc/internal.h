@@ -51,6 +51,8 @@ cudaError_t launch_prefill(const LaunchArgs& a);
 int prefill_rows_per_thread(int64_t M);
 // Fixed-order RMSNorm of M rows of H elements (rmsnorm.cu).
 cudaError_t launch_rmsnorm(const float* x, const float* g, float eps, int64_t M, int64_t H, float* y, cudaStream_t stream);
+// Read `bytes` at buf through L2 (evicts what was there without leaving dirty lines); sink: 4 bytes of device memory.
+cudaError_t launch_l2_evict(const void* buf, size_t bytes, unsigned* sink, int sm_count, cudaStream_t stream);
 cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cudaStream_t stream);
 
 // Decode-kernel tiling chosen for a shape (numerically inert); used by the host to build the
@@ -62,6 +64,8 @@ struct DecodeConfig {
 // S = number of K segments of the order (it only scales the unit count in the schedule's cost model)
 bool decode_config_for(int64_t M, int64_t N, int64_t K, int S, int wfmt, int variant, DecodeConfig* out);
 int decode_num_variants();
+// resident blocks per SM of a tiling on the current device (schedule information only)
+int decode_config_occupancy(int wfmt, const DecodeConfig& cfg);
 
 }  // namespace detlin
 

@@ -101,6 +101,11 @@ bool decode_config_for(int64_t M, int64_t N, int64_t K, int S, int wfmt, int var
     return true;
 }
 
+int decode_config_occupancy(int wfmt, const DecodeConfig& cfg)
+{
+    return class_table(wfmt, cfg.id / 64)->entries[cfg.id % 64].occupancy();
+}
+
 cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
 {
     DecodeConfig cfg;

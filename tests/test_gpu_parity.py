@@ -211,3 +211,33 @@ def test_prefill_tile_choice():
     with pytest.raises(B.DetLinearError):
         B.det_test_plan_set_variant(plan, 3)
     plan.close()
+
+
+def test_plan_tune_changes_the_schedule_only():
+    """det_linear_plan_tune pins the fastest tiling; the bits before and after are the oracle's."""
+    for (M, N, K) in ((2, 6144, 4096), (8, 1000, 1024), (24, 4096, 4096)):
+        x, W, b = inputs.make_case(M, N, K)
+        xd, Wd, bd = x.cuda(), W.cuda(), b.cuda()
+        y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        plan = B.det_linear_plan(M, N, K)
+        B.det_linear_run(plan, xd, Wd, bd, y)
+        torch.cuda.synchronize()
+        before = y.cpu().numpy()
+        variant, us = B.det_linear_plan_tune(plan, xd, Wd, bd, y)
+        assert variant >= 1 and us > 0
+        d = B.det_linear_plan_describe(plan)
+        assert d["variant"] == variant and d["decode_tiling"]["blocks_per_sm"] >= 1
+        y.fill_(float("nan"))
+        B.det_linear_run(plan, xd, Wd, bd, y)
+        B.det_linear_plan_check(plan)
+        after = y.cpu().numpy()
+        plan.close()
+        if N * K <= 4096 * 4096 and M <= 8:
+            assert_bits_equal(before, oracle_y(x, W, b), f"before {M},{N},{K}")
+        assert_bits_equal(after, before, f"after tuning {M},{N},{K}")
+    # nothing to choose in the prefill bucket
+    x, W, b = inputs.make_case(100, 256, 512)
+    plan = B.det_linear_plan(100, 256, 512)
+    y = torch.empty(100, 256, device="cuda")
+    assert B.det_linear_plan_tune(plan, x.cuda(), W.cuda(), b.cuda(), y) == (0, -1.0)
+    plan.close()
