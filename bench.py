@@ -691,8 +691,26 @@ def cpu_baseline(work):
 def run_case(args):
     """One shape, few launches: the workload used for ncu captures of a single kernel."""
     from paper_2609_25624_b200 import binding as B
-    M, N, K = (int(v) for v in args.case.split(","))
+    dims = [int(v) for v in args.case.split(",")]
     torch.cuda.set_device(0)
+    if len(dims) == 2:                       # M,H: the fixed-order RMSNorm kernel
+        M, H = dims
+        x = torch.randn(M, H, generator=torch.Generator().manual_seed(M)).cuda()
+        g = torch.ones(H, device="cuda")
+        y = torch.empty_like(x)
+        for _ in range(3):
+            B.det_rmsnorm(x, g, 1e-5, y)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            B.det_rmsnorm(x, g, 1e-5, y)
+        e1.record()
+        torch.cuda.synchronize()
+        print(json.dumps({"case": ["rmsnorm", M, H], "launches": args.steps, "warmup_launches": 3,
+                          "us_per_launch_eager": e0.elapsed_time(e1) * 1e3 / args.steps}), flush=True)
+        return
+    M, N, K = dims
     x, W, b = inputs.make_case(M, N, K)
     copies = max(2, min(8, -(-(256 << 20) // (2 * N * K))))       # > L2 in total, a few hundred MB at most
     Ws = [W.cuda()] + [W.cuda().clone() for _ in range(copies - 1)]
@@ -723,8 +741,8 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-case, prefill and LM-head tables")
     ap.add_argument("--ref-cols", type=int, default=512, help="weight rows per case in the reference arm's sample")
-    ap.add_argument("--case", default=None, metavar="M,N,K",
-                    help="run only this shape: --steps eager det_linear_run calls over rotating weight copies "
+    ap.add_argument("--case", default=None, metavar="M,N,K | M,H",
+                    help="M,H: a few det_rmsnorm launches.  M,N,K: run only this shape: --steps eager det_linear_run calls over rotating weight copies "
                          "(a small, profiler-friendly workload; prints its own one-line JSON)")
     args = ap.parse_args()
     if args.case:

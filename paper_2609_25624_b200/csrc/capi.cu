@@ -251,12 +251,11 @@ det_status_t det_rmsnorm(const float* x, const float* g, float eps, int64_t M, i
         return DET_ERR_INVALID_ARG;
     }
     if (!(eps >= 0.0f)) { set_error("rmsnorm: eps must be a non-negative number"); return DET_ERR_INVALID_ARG; }
-    int dev = 0;
-    cudaDeviceProp prop;
+    int dev = 0, major = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);   // cheap, per call
     if (e != cudaSuccess) return cuda_fail("rmsnorm: device query", e);
-    if (prop.major != 10) { set_error("rmsnorm: device %d is sm_%d%d; this library is built for sm_100a only", dev, prop.major, prop.minor); return DET_ERR_ARCH; }
+    if (major != 10) { set_error("rmsnorm: device %d is sm_%dx; this library is built for sm_100a only", dev, major); return DET_ERR_ARCH; }
     e = launch_rmsnorm(x, g, eps, M, H, y, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail("rmsnorm: launch", e);
     return DET_OK;

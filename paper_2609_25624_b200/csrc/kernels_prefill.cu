@@ -80,6 +80,7 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
     constexpr int TB = TR - 4;                       // rows of a thread in the upper group (1 .. 4)
     constexpr int XP = (BM * 8 + 255) / 256;         // 16-byte pieces of x per thread and slab
     const int tid = threadIdx.x;
+    // 16 x 16 threads; a warp = 16 column groups x 2 row groups (8 x 4 and 4 x 8 warps measured 7 % slower)
     const int tx = tid & 15, ty = tid >> 4;
 
     // block -> (m tile fastest, then n tile, then segment)
