@@ -670,22 +670,27 @@ def layercast_table(work, st, per_case):
 
 
 def cpu_baseline(work):
-    """The oracle as it stands, on the host cores, on a bounded sample of the same step."""
+    """The oracle as it stands, on the host cores, on a bounded sample of the same step: every case of
+    the sweep restricted to its first 8192 weight rows (all rows for N <= 8192), five passes (about
+    ten seconds of host time on 16 cores)."""
     from oracle import oracle
-    cols = 512
+    cap, passes = 8192, 5
     data = []
+    sample_bytes = 0
     for w in work:
-        xs = w["xh"].numpy()
-        Wb = inputs.bf16_bits(w["W"][:cols].cpu())
-        data.append((xs, Wb, w["b"][:cols].cpu().numpy(), oracle.order_params(w["M"], w["N"], w["K"])))
-    oracle.linear(*data[0][:3], params=data[0][3])          # load the library
+        rows = min(w["N"], cap)
+        Wb = inputs.bf16_bits(w["W"][:rows].cpu())
+        data.append((w["xh"].numpy(), Wb, w["b"][:rows].cpu().numpy(), oracle.order_params(w["M"], w["N"], w["K"])))
+        sample_bytes += 2 * rows * w["K"]
+    oracle.linear(data[0][0], data[0][1][:64], data[0][2][:64], params=data[0][3])          # load the library
     t0 = time.perf_counter()
-    for x, Wb, b, prm in data:
-        oracle.linear(x, Wb, b, params=prm)
-    dt = time.perf_counter() - t0
-    sample_bytes = sum(2 * cols * w["K"] for w in work)
+    for _ in range(passes):
+        for x, Wb, b, prm in data:
+            oracle.linear(x, Wb, b, params=prm)
+    dt = (time.perf_counter() - t0) / passes
     return {"value": sample_bytes / dt / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": f"all 20 cases of the step, first {cols} of N weight rows each (one pass, {dt:.2f} s)"}
+            "sample": f"all 20 cases of the step, first {cap} weight rows of each (all rows when N <= {cap}), "
+                      f"{passes} passes of {dt:.2f} s"}
 
 
 def run_case(args):
@@ -740,7 +745,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-case, prefill and LM-head tables")
-    ap.add_argument("--ref-cols", type=int, default=512, help="weight rows per case in the reference arm's sample")
+    ap.add_argument("--ref-cols", type=int, default=2048, help="weight rows per case in the reference arm's sample")
     ap.add_argument("--case", default=None, metavar="M,N,K | M,H",
                     help="M,H: a few det_rmsnorm launches.  M,N,K: run only this shape: --steps eager det_linear_run calls over rotating weight copies "
                          "(a small, profiler-friendly workload; prints its own one-line JSON)")
