@@ -467,8 +467,13 @@ template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG, int WF>
 int decode_occupancy_t()
 {
     using C = Cfg<MT, WM, RT, WR, KC, STAGES, PG, WF>;
-    static int blocks_per_sm = -1;
-    if (blocks_per_sm < 0) {
+    // function attributes belong to a device: opt in to the large shared-memory carve-out and cache
+    // the answer once per device (benign if two threads race: both store the same value)
+    static int blocks_per_sm[kMaxDevices];
+    static bool known[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return 0; }
+    if (!known[dev]) {
         auto kern = decode_kernel<MT, WM, RT, WR, KC, STAGES, PG, WF>;
         int occ = 0;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess ||
@@ -476,9 +481,10 @@ int decode_occupancy_t()
             cudaGetLastError();
             return 0;
         }
-        blocks_per_sm = occ;
+        blocks_per_sm[dev] = occ;
+        known[dev] = true;
     }
-    return blocks_per_sm;
+    return blocks_per_sm[dev];
 }
 
 template <int MT, int WM, int RT, int WR, int KC, int STAGES, int PG, int WF>

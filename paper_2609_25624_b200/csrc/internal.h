@@ -20,6 +20,8 @@ struct DeviceStatus {
     unsigned int where;          // which wait (diagnostic)
 };
 
+constexpr int kMaxDevices = 64;     // per-device caches (function attributes, symbol addresses)
+
 void set_error(const char* fmt, ...);
 det_status_t fill_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* out);
 

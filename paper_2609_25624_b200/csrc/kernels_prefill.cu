@@ -259,11 +259,15 @@ template <int WF, int TR>
 cudaError_t launch_prefill_t(const LaunchArgs& a)
 {
     constexpr int BM = 16 * TR;
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices];             // function attributes belong to a device
+    int dev = 0;
+    cudaError_t de = cudaGetDevice(&dev);
+    if (de != cudaSuccess) return de;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(prefill_kernel<WF, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
     const int tiles_m = (int)((a.M + BM - 1) / BM), tiles_n = (int)((a.N + BN - 1) / BN);
     const long long units = (long long)tiles_m * tiles_n * a.S;

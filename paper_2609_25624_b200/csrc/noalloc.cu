@@ -19,7 +19,6 @@ namespace detlin {
 constexpr size_t kNoallocScratchFloats = (size_t)1 << 20;
 static __device__ __align__(256) float g_noalloc_scratch[kNoallocScratchFloats];
 
-constexpr int kMaxDevices = 64;
 static float* g_scratch_addr[kMaxDevices];      // device address of the array, per device
 static std::mutex g_scratch_mutex;
 
