@@ -60,6 +60,15 @@ DET_API det_status_t det_test_measure_read_bandwidth(const void* buf, size_t byt
 DET_API det_status_t det_test_linear_atomic_splitk(int64_t M, int64_t N, int64_t K, int32_t S_req, const float* x,
                                                    const uint16_t* W, const float* b, float* y, void* stream);
 
+/*
+ * Glue for the multi-layer test harness (no part of the method): dst[m, j] = src[m, j] * c for the first
+ * `cols` columns of a row-major device matrix with row pitch ld_src; dst is [M, cols], contiguous.
+ * One IEEE multiplication per element.  Enqueued on `stream` with programmatic dependent launch, so a
+ * chain det_linear_run -> glue -> det_linear_run keeps overlapping kernel prologues.
+ */
+DET_API det_status_t det_test_scale_cols(const float* src, int64_t ld_src, float* dst, int64_t M, int64_t cols, float c,
+                                         void* stream);
+
 #ifdef __cplusplus
 }
 #endif

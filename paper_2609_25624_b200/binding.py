@@ -94,6 +94,8 @@ def lib() -> ctypes.CDLL:
         L.det_linear_run_noalloc.restype = i32
         L.det_test_linear_atomic_splitk.argtypes = [i64, i64, i64, ctypes.c_int32, p, p, p, p, p]
         L.det_test_linear_atomic_splitk.restype = i32
+        L.det_test_scale_cols.argtypes = [p, i64, p, i64, i64, ctypes.c_float, p]
+        L.det_test_scale_cols.restype = i32
         L.det_test_measure_fma_peak.argtypes = [i32, ctypes.POINTER(ctypes.c_double)]
         L.det_test_measure_fma_peak.restype = i32
         L.det_test_measure_read_bandwidth.argtypes = [p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_double)]
@@ -365,3 +367,12 @@ def det_test_linear_atomic_splitk(x, W, b, y, S_req: int, stream=None) -> None:
         _expect(b, torch.float32, (N,), "b")
     _check(lib().det_test_linear_atomic_splitk(M, N, K, int(S_req), x.data_ptr(), W.data_ptr(),
                                                b.data_ptr() if b is not None else None, y.data_ptr(), _stream_ptr(stream)))
+
+
+def det_test_scale_cols(src, cols: int, c: float, stream=None):
+    """Harness glue: returns a new contiguous [M, cols] tensor = src[:, :cols] * c (one rounding each)."""
+    M, ld = src.shape
+    _expect(src, torch.float32, (M, ld), "src")
+    dst = torch.empty((M, cols), dtype=torch.float32, device=src.device)
+    _check(lib().det_test_scale_cols(src.data_ptr(), ld, dst.data_ptr(), M, cols, float(c), _stream_ptr(stream)))
+    return dst

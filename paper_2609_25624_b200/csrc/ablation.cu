@@ -44,9 +44,45 @@ atomic_splitk_kernel(const float* __restrict__ x, const uint16_t* __restrict__ W
     }
 }
 
+// Harness glue for multi-layer tests: dst[m, j] = src[m, j] * c for the first `cols` columns of a
+// row-major matrix with row pitch ld_src (one rounding per element).  Launched with programmatic
+// dependent launch on both sides so that a chain linear -> glue -> linear keeps overlapping.
+__global__ void __launch_bounds__(256)
+scale_cols_kernel(const float* __restrict__ src, int64_t ld_src, float* __restrict__ dst, int64_t M, int64_t cols, float c)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int64_t total = M * cols;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t m = i / cols, j = i - m * cols;
+        dst[i] = __fmul_rn(src[m * ld_src + j], c);
+    }
+}
+
 }  // namespace detlin
 
 using namespace detlin;
+
+extern "C" det_status_t det_test_scale_cols(const float* src, int64_t ld_src, float* dst, int64_t M, int64_t cols, float c,
+                                            void* stream)
+{
+    if (!src || !dst || M < 1 || cols < 1 || ld_src < cols) { set_error("scale_cols: bad argument"); return DET_ERR_INVALID_ARG; }
+    const int64_t total = M * cols;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, scale_cols_kernel, src, ld_src, dst, M, cols, c);
+    if (e != cudaSuccess) { set_error("scale_cols: launch failed: %s", cudaGetErrorString(e)); return DET_ERR_CUDA; }
+    return DET_OK;
+}
 
 extern "C" det_status_t det_test_linear_atomic_splitk(int64_t M, int64_t N, int64_t K, int32_t S_req, const float* x,
                                                       const uint16_t* W, const float* b, float* y, void* stream)

@@ -149,6 +149,10 @@ argmax_rows_kernel(const float* __restrict__ y, int64_t N, int32_t* __restrict__
     __shared__ int si[32];
     __shared__ float block_v;
     __shared__ int block_i;
+    // programmatic dependent launch: let the next kernel of the stream start its prologue now, and
+    // wait for the kernel that produced y before reading it
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const float* row = y + (int64_t)blockIdx.y * N;
@@ -191,10 +195,20 @@ cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cu
     const int64_t max_rows = 65535;
     for (int64_t m0 = 0; m0 < M; m0 += max_rows) {
         const int64_t mm = (M - m0 < max_rows) ? M - m0 : max_rows;
-        dim3 grid(kArgmaxCluster, (unsigned)mm);
-        argmax_rows_kernel<<<grid, 1024, 0, stream>>>(y + m0 * N, N, idx + m0);
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(kArgmaxCluster, (unsigned)mm);
+        cfg.blockDim = dim3(1024);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, argmax_rows_kernel, y + m0 * N, N, idx + m0);
+        if (e != cudaSuccess) return e;
     }
-    return cudaGetLastError();
+    return cudaSuccess;
 }
 
 }  // namespace detlin

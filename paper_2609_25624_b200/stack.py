@@ -2,7 +2,8 @@
 
 32 layers x (qkv 4096->6144, o 4096->4096, gate_up 4096->28672, down 14336->4096) + LM head
 4096->128256, about 15 GB of BF16 weights.  Only the linear layers are the library's kernels; the
-glue between them is elementwise (slice, multiply by a constant, gather), chosen so that nothing
+glue between them is elementwise (slice, multiply by a constant -- a test-only kernel that keeps the
+programmatic-dependent-launch chain intact -- and a gather), chosen so that nothing
 order-dependent is introduced and the activations stay near N(0, 1):
 
     q  = c1 * qkv(x)[:, :4096]        c1 = c2 = c3 = 1 / (0.02 * sqrt(4096))
@@ -93,19 +94,19 @@ class LinearStack:
         y = self.linear(plans, "qkv", w["qkv"], x, stream)
         if trace is not None:
             trace(layer, "qkv", x, y)
-        q = (y[:, :HIDDEN] * float(C_IN)).contiguous()
+        q = B.det_test_scale_cols(y, HIDDEN, float(C_IN), stream)
         y = self.linear(plans, "o", w["o"], q, stream)
         if trace is not None:
             trace(layer, "o", q, y)
-        o = y * float(C_IN)
+        o = B.det_test_scale_cols(y, HIDDEN, float(C_IN), stream)
         y = self.linear(plans, "gate_up", w["gate_up"], o, stream)
         if trace is not None:
             trace(layer, "gate_up", o, y)
-        h = (y[:, :FFN] * float(C_IN)).contiguous()
+        h = B.det_test_scale_cols(y, FFN, float(C_IN), stream)
         y = self.linear(plans, "down", w["down"], h, stream)
         if trace is not None:
             trace(layer, "down", h, y)
-        return y * float(C_DOWN)
+        return B.det_test_scale_cols(y, HIDDEN, float(C_DOWN), stream)
 
     def step(self, plans, x, stream=None, trace=None):
         """One decode step: x [M, 4096] -> (logits [M, 128256], argmax [M] int32, next x)."""
