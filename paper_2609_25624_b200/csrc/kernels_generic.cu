@@ -68,6 +68,10 @@ __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ partials, const float* __restrict__ b, float* __restrict__ y,
                int64_t MN, int64_t N, int S, int64_t ldy)
 {
+    // programmatic dependent launch: the next kernel may start its prologue; the partials are read
+    // only after the kernel that wrote them has completed
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= MN) return;
     float t = partials[i];
@@ -113,8 +117,16 @@ cudaError_t launch_generic(const LaunchArgs& a, int bucket)
 cudaError_t launch_combine(const LaunchArgs& a)
 {
     const int64_t MN = a.M * a.N;
-    combine_kernel<<<(unsigned)((MN + 255) / 256), 256, 0, a.stream>>>(a.partials, a.b, a.y, MN, a.N, a.S, a.ldy);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)((MN + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, combine_kernel, (const float*)a.partials, a.b, a.y, MN, a.N, a.S, a.ldy);
 }
 
 // Row argmax, lowest index on ties (the paper's stated tie rule for greedy decoding).  Ordering
