@@ -100,3 +100,19 @@ def test_sixty_four_steps_bitwise_identical_across_runs_streams_and_sm_limits(st
             B.det_test_plan_set_max_blocks(p, 24)
         d3, t3 = st.run(x0, 16, key="capped")
     assert d3 == ref_digests[:16] and t3 == ref_tokens[:16]
+
+
+def test_harness_glue_kernel_matches_the_plain_elementwise_definition():
+    """det_test_scale_cols (the harness's slice-and-rescale step) is one IEEE multiplication per
+    element: it must equal the same product computed by torch, bit for bit, for any pitch."""
+    import numpy as np
+    import torch
+    from paper_2609_25624_b200 import binding as B
+    g = torch.Generator().manual_seed(21)
+    for (M, ld, cols, c) in ((1, 6144, 4096, 0.78125), (8, 28672, 14336, 0.41762), (5, 37, 13, -3.3), (64, 128, 128, 1e-3)):
+        src = torch.randn(M, ld, generator=g).cuda()
+        got = B.det_test_scale_cols(src, cols, c)
+        want = src[:, :cols] * torch.tensor(c, dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        assert got.shape == (M, cols)
+        assert np.array_equal(got.cpu().numpy().view(np.uint32), want.cpu().numpy().view(np.uint32)), (M, ld, cols)
