@@ -94,10 +94,13 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
     const int k_hi = min(K, k_lo + seg_len);
 
     // ---- staging assignment (global rows are k-contiguous, shared tiles are k-major: a transpose) ----
-    // x tile: BM rows x 8 quads (4 floats = 16 bytes).  Piece p = tid + 256 j: half o = p & 1,
-    //   row r = (p >> 1) mod BM, quad q = 2 * ((p >> 1) / BM) + o.  Two neighbouring lanes read one 32-byte
-    //   sector; the four scalar stores of a lane go to k rows 4q .. 4q+3, conflict-free across the warp
-    //   (bank = 16 o + 4 e + r mod 32 over 16 consecutive r and o in {0, 1}).
+    // x tile: BM rows x 8 quads (4 floats = 16 bytes).  Piece p = tid + 256 j: o = p & 3,
+    //   row r = (p >> 2) mod BM, quad q = 4 * ((p >> 2) / BM) + o.  Four neighbouring lanes read 64
+    //   contiguous bytes of a row, so a warp's load touches 8 rows (with two lanes per row and 16 rows
+    //   per load the kernel measured 4 % slower; with eight lanes per row 6 % slower again because of
+    //   four-way store conflicts).  The four scalar stores of a lane go to k rows 4q .. 4q+3, two-way
+    //   bank conflicts (bank = 16 o + 4 e + r mod 32 over o in 0..3 and 8 consecutive r); a column
+    //   swizzle that removes them cost more in the multiply loop than it saved.
     // w tile: 128 rows x 4 octets (8 BF16 = 16 bytes).  Piece p = tid + 256 j: half o = p & 1,
     //   row r = (p >> 1) & 127, octet c = 2 * (p >> 8) + o; eight scalar stores to k rows 8c .. 8c+7
     //   (two-way bank conflicts between the two halves; 16 stores per thread and slab).
@@ -108,7 +111,7 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
 #pragma unroll
     for (int j = 0; j < XP; ++j) {
         const int p = tid + 256 * j;
-        const int o = p & 1, r = (p >> 1) % BM, q = 2 * ((p >> 1) / BM) + o;
+        const int o = p & 3, r = (p >> 2) % BM, q = 4 * ((p >> 2) / BM) + o;
         const int m = m0 + r;
         xok[j] = m < M && p < BM * 8;
         xk[j] = q * 4;
