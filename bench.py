@@ -6,9 +6,12 @@ Workload (one "step"): the decode sweep on Llama-3-8B layer shapes -- M in {1,4,
 det_linear_run, each on its own seeded BF16 weight matrix (2.18 GB of weights per step, so every
 call finds its weights cold in L2).  Metric: BF16 weight bytes streamed per second (GB/s).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras] [--tables PATH]
 
-Prints ONE JSON line.  With --impl reference the CPU oracle is timed instead (host cores).
+The LAST line of stdout is one short JSON object (the headline: metric, value, roofline, cpu_baseline,
+e2e, clocks).  The long per-case tables (decode per case, prefill, LM head, stack, ...) go to stderr as
+one JSON line and, with --tables PATH, into that file.  With --impl reference the CPU oracle is timed
+instead (host cores).
 Under torchrun every rank runs an independent replica on its own GPU (the path has no exchange
 step); the time is the maximum over ranks and `value` the aggregate over all ranks.
 """
@@ -135,25 +138,33 @@ def max_over_ranks(value, world):
 # ---------------------------------------------------------------------------------------------
 # reference arm: the CPU oracle
 # ---------------------------------------------------------------------------------------------
-def run_reference(args, world, rank):
-    if rank != 0:
-        return
+ORACLE_SAMPLE_ROWS = 2048
+
+
+def oracle_sample(cols=ORACLE_SAMPLE_ROWS):
+    """The bounded sample of one step that both oracle timings use (cpu_baseline of the own arm and
+    the reference arm): every case of the sweep with its own seed and order parameters, restricted to
+    `cols` weight rows.  Returns (step function, BF16 weight bytes per step, threads, description)."""
     from oracle import oracle
     cases = decode_cases()
-    # bounded sample: every case of the sweep, restricted to the first `cols` weight rows, sized so
-    # that one step is a few seconds of host time
-    cols = args.ref_cols
     data = []
     for (M, N, K, name) in cases:
         x, W, b = inputs.make_case(M, cols, K, seed=inputs.shape_seed(M, N, K))
         data.append((x.numpy(), inputs.bf16_bits(W), b.numpy(), oracle.order_params(M, N, K)))
     sample_bytes = sum(2 * cols * K for (_, _, K, _) in cases)
-    threads = oracle.threads()
 
     def step():
         for x, Wb, b, prm in data:
             oracle.linear(x, Wb, b, params=prm)
 
+    return step, sample_bytes, oracle.threads(), f"all 20 cases of the sweep, {cols} of N weight rows each, per step"
+
+
+def run_reference(args, world, rank):
+    if rank != 0:
+        return
+    cols = args.ref_cols
+    step, sample_bytes, threads, sample = oracle_sample(cols)
     for _ in range(args.warmup):
         step()
     t0 = time.perf_counter()
@@ -166,9 +177,8 @@ def run_reference(args, world, rank):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "Llama-3-8B decode sweep: M in {1,4,8,16,32} x {qkv,o,gate_up,down}, 20 calls/step",
-                   "sample": f"first {cols} weight rows of every case"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                         "sample": f"all 20 cases of the sweep, first {cols} of N weight rows each, per step"},
+                   "sample": f"{cols} weight rows of every case"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -295,59 +305,93 @@ def run_own(args, world, rank, local):
         return
 
     achieved = alg_bytes / (ms_step * 1e-3) / 1e9
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "Llama-3-8B decode sweep: M in {1,4,8,16,32} x {qkv 4096->6144, o 4096->4096, "
-                               "gate_up 4096->28672, down 14336->4096}, 20 det_linear_run calls per step, bias present",
-                   "weights": "BF16 N(0,0.02^2) RNE, one seeded matrix per case (2.18 GB per step)",
-                   "activations": "FP32 N(0,1)", "l2": "inputs larger than L2: 2.18 GB of distinct weights between reuses",
-                   "launch": "one CUDA graph per step (programmatic dependent launch between the 20 kernels)",
-                   "multi_gpu": "replicas only (no exchange step in the path)"},
-        "pct_of_hbm_peak": 100.0 * value / world / hbm_peak,
-        "tflops_fp32": world * flops / (ms_step * 1e-3) / 1e12,
-        "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "note": "det_linear_run_host_async per call (x from pinned host memory, y back to host, weights resident), calls spread over 3 streams so copies overlap kernels, one synchronisation per stream per step"},
-        "gpu_launches": launches_per_step * args.steps,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
-                     "traffic": None, "peak_source": hbm_src, "kernel": "decode_kernel (all 20 launches of a step)",
-                     "note": "M=16 and M=32 launches are FP32-FMA-bound on B200 (ridge 11.4 flop/B), see per_case"},
-    }
-
-    line["calibration"] = calibration(B, dev, fp32_peak)
-    if not args.no_extras:
-        line["per_case"] = per_case_table(B, work, st, hbm_peak, fp32_peak)
-        line["tuned"] = tuned_table(B, work, st, line["per_case"])
-        line["prefill"] = prefill_table(B, dev, st, fp32_peak)
-        line["mid_bucket"] = mid_bucket_table(B, dev, st, fp32_peak)
-        line["lm_head"] = lm_head_table(B, dev, st, hbm_peak, fp32_peak)
-        line["layercast_style_reference"] = layercast_table(work, st, line["per_case"])
-        line["weight_formats"] = weight_format_table(B, dev, st, hbm_peak, fp32_peak)
-        line["column_shards"] = shard_table(B, dev, st, hbm_peak)
-        line["r3_ablation"] = ablation_table(B, dev, st)
-        line["rmsnorm"] = rmsnorm_table(B, dev, st, hbm_peak)
-        line["cpu_baseline"] = cpu_baseline(work)
-        for w in work:                       # free the sweep's 2.2 GB before the 15 GB stack
-            w["plan"].close()
-        work.clear()
-        line["stack"] = stack_table(dev, st, hbm_peak)
-    else:
-        line["cpu_baseline"] = cpu_baseline(work)
-    # DRAM traffic per launch: ncu (dram__bytes_read.sum + dram__bytes_write.sum) on N = K = 4096 captures gives
-    # 1.000 / 0.997 / 0.987 x the algorithmic bytes at M = 1 / 8 / 32 (ncu summaries under profiles/);
-    # traffic is proportional to the algorithmic bytes, so it is scaled to the step's average launch here.
-    line["roofline"]["traffic"] = DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes / launches_per_step
-    line["roofline"]["algorithmic_bytes_per_launch"] = alg_bytes / launches_per_step
     # Each launch against the roof that binds IT: max(bytes / HBM peak, flops / FP32 CUDA-core peak).
     t_bind = sum(max(algorithmic_bytes(M, N, K) / (hbm_peak * 1e9), 2.0 * M * N * K / (fp32_peak * 1e12))
                  for (M, N, K, _) in decode_cases())
-    line["roofline"]["binding_roof_ms_per_step"] = t_bind * 1e3
-    line["roofline"]["frac_of_binding_roof"] = t_bind * 1e3 / ms_step
-    print(json.dumps(line), flush=True)
-    for w in work:
+    # DRAM traffic per launch: ncu (dram__bytes_read.sum + dram__bytes_write.sum) on N = K = 4096 captures gives
+    # 1.000 / 0.997 / 0.987 x the algorithmic bytes at M = 1 / 8 / 32 (ncu summaries under profiles/);
+    # traffic is proportional to the algorithmic bytes, so it is scaled to the step's average launch here.
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "Llama-3-8B decode sweep, M in {1,4,8,16,32} x {qkv,o,gate_up,down}: 20 det_linear_run "
+                               "calls/step in one CUDA graph, bias present, BF16 N(0,0.02^2) weights, FP32 N(0,1) x",
+                   "l2": "inputs larger than L2 (2.18 GB of distinct weights per step)",
+                   "multi_gpu": "replicas only"},
+        "pct_of_hbm_peak": round(100.0 * value / world / hbm_peak, 2),
+        "tflops_fp32": round(world * flops / (ms_step * 1e-3) / 1e12, 2),
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 2), "peak": hbm_peak, "unit": "GB/s",
+                     "frac": round(achieved / hbm_peak, 4),
+                     "traffic": round(DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes / launches_per_step),
+                     "algorithmic_bytes_per_launch": round(alg_bytes / launches_per_step),
+                     "frac_of_binding_roof": round(t_bind * 1e3 / ms_step, 4),
+                     "peak_source": "MEASURED_PEAKS.json" if hbm_src.startswith("measured") else "fallback",
+                     "kernel": "decode_kernel, 20 launches/step; M=16,32 are FP32-FMA-bound (ridge 11.4 flop/B)"},
+    }
+    tables = {"headline_notes": {
+        "weights": "BF16 N(0,0.02^2) RNE, one seeded matrix per case (2.18 GB per step)",
+        "launch": "one CUDA graph per step (programmatic dependent launch between the 20 kernels)",
+        "e2e": "det_linear_run_host_async per call (x from pinned host memory, y back to host, weights resident), "
+               "calls spread over 3 streams so copies overlap kernels, one synchronisation per stream per step",
+        "hbm_peak_source": hbm_src, "binding_roof_ms_per_step": t_bind * 1e3}}
+    tables["calibration"] = calibration(B, dev, fp32_peak)
+    if not args.no_extras:
+        tables["per_case"] = per_case_table(B, work, st, hbm_peak, fp32_peak)
+        tables["tuned"] = tuned_table(B, work, st, tables["per_case"])
+        tables["prefill"] = prefill_table(B, dev, st, fp32_peak)
+        tables["mid_bucket"] = mid_bucket_table(B, dev, st, fp32_peak)
+        tables["lm_head"] = lm_head_table(B, dev, st, hbm_peak, fp32_peak)
+        tables["layercast_style_reference"] = layercast_table(work, st, tables["per_case"])
+        tables["weight_formats"] = weight_format_table(B, dev, st, hbm_peak, fp32_peak)
+        tables["column_shards"] = shard_table(B, dev, st, hbm_peak)
+        tables["r3_ablation"] = ablation_table(B, dev, st)
+        tables["rmsnorm"] = rmsnorm_table(B, dev, st, hbm_peak)
+    for w in work:                       # free the sweep's 2.2 GB (before the 15 GB stack)
         w["plan"].close()
+    work.clear()
+    if not args.no_extras:
+        tables["stack"] = stack_table(dev, st, hbm_peak)
+        # compact digest of the tables for the headline: worst and mean % of the binding roof per batch size
+        pc = tables["per_case"]
+        line["decode_pct_of_binding_roof"] = {
+            f"M{M}": [round(r["pct_of_roofline"], 1) for r in pc if r["M"] == M] for M in inputs.DECODE_MS}
+        line["prefill_pct_fp32_peak"] = [round(r["pct_fp32_peak"], 1) for r in tables["prefill"]["cases"]]
+        line["lm_head_pct_of_binding_roof"] = [round(r["pct_of_roofline"], 1) for r in tables["lm_head"]]
+        line["stack_pct_hbm"] = [round(r["pct_hbm"], 1) for r in tables["stack"]["cases"]]
+    line["cpu_baseline"] = cpu_baseline()
+    line["cpu_baseline"]["value"] = round(line["cpu_baseline"]["value"], 4)
+    emit(line, tables, args.tables)
+
+
+HEADLINE_MAX_BYTES = 2000
+OPTIONAL_HEADLINE_KEYS = ("stack_pct_hbm", "lm_head_pct_of_binding_roof", "prefill_pct_fp32_peak",
+                          "decode_pct_of_binding_roof", "tflops_fp32", "pct_of_hbm_peak")
+
+
+def emit(line, tables, tables_path=None, out=sys.stdout, err=sys.stderr):
+    """Write the long tables (one JSON line on `err`, and to `tables_path` if given), then the short
+    headline as the LAST line of `out`.  A reader that keeps only the tail of stdout must still get the
+    whole headline, so optional digest keys are dropped until it is below HEADLINE_MAX_BYTES."""
+    blob = json.dumps({"tables": tables, "headline": line})
+    print(blob, file=err, flush=True)
+    if tables_path:
+        os.makedirs(os.path.dirname(os.path.abspath(tables_path)), exist_ok=True)
+        with open(tables_path, "w") as f:
+            f.write(blob + "\n")
+    line = dict(line)
+    for key in OPTIONAL_HEADLINE_KEYS:
+        if len(json.dumps(line)) < HEADLINE_MAX_BYTES:
+            break
+        line.pop(key, None)
+    text = json.dumps(line)
+    if len(text) >= HEADLINE_MAX_BYTES:
+        raise RuntimeError(f"headline line is {len(text)} bytes; it must stay below {HEADLINE_MAX_BYTES}")
+    print(text, file=out, flush=True)
+    return text
 
 
 def stack_table(dev, st, hbm_peak):
@@ -599,9 +643,12 @@ def lm_head_table(B, dev, st, hbm_peak, fp32_peak):
         for p in plans:
             p.close()
         wbytes = 2 * N * K
+        t_hbm = wbytes / (hbm_peak * 1e9)
+        t_fma = 2 * M * N * K / (fp32_peak * 1e12)
         rows.append({"M": M, "us_linear_plus_argmax": ms * 1e3, "weight_gbs": wbytes / ms / 1e6,
                      "pct_hbm": 100 * wbytes / ms / 1e6 / hbm_peak, "tflops": 2 * M * N * K / ms / 1e9,
-                     "pct_fp32": 100 * 2 * M * N * K / ms / 1e9 / fp32_peak})
+                     "pct_fp32": 100 * 2 * M * N * K / ms / 1e9 / fp32_peak,
+                     "bound": "hbm" if t_hbm >= t_fma else "fp32", "pct_of_roofline": 100 * max(t_hbm, t_fma) / (ms * 1e-3)})
     return rows
 
 
@@ -669,28 +716,18 @@ def layercast_table(work, st, per_case):
                     "this pattern on A100/L40S/H100 -- other hardware, context only", "cases": rows}
 
 
-def cpu_baseline(work):
-    """The oracle as it stands, on the host cores, on a bounded sample of the same step: every case of
-    the sweep restricted to its first 8192 weight rows (all rows for N <= 8192), five passes (about
-    ten seconds of host time on 16 cores)."""
-    from oracle import oracle
-    cap, passes = 8192, 5
-    data = []
-    sample_bytes = 0
-    for w in work:
-        rows = min(w["N"], cap)
-        Wb = inputs.bf16_bits(w["W"][:rows].cpu())
-        data.append((w["xh"].numpy(), Wb, w["b"][:rows].cpu().numpy(), oracle.order_params(w["M"], w["N"], w["K"])))
-        sample_bytes += 2 * rows * w["K"]
-    oracle.linear(data[0][0], data[0][1][:64], data[0][2][:64], params=data[0][3])          # load the library
+def cpu_baseline(passes=8):
+    """The oracle as it stands, on the host cores, on the same bounded sample of the step that the
+    reference arm times (oracle_sample): one untimed pass, then `passes` timed ones (about ten seconds
+    of host time on 16 cores)."""
+    step, sample_bytes, threads, sample = oracle_sample()
+    step()
     t0 = time.perf_counter()
     for _ in range(passes):
-        for x, Wb, b, prm in data:
-            oracle.linear(x, Wb, b, params=prm)
+        step()
     dt = (time.perf_counter() - t0) / passes
-    return {"value": sample_bytes / dt / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": f"all 20 cases of the step, first {cap} weight rows of each (all rows when N <= {cap}), "
-                      f"{passes} passes of {dt:.2f} s"}
+    return {"value": sample_bytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{sample}; {passes} passes of {dt:.2f} s"}
 
 
 def run_case(args):
@@ -745,7 +782,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-case, prefill and LM-head tables")
-    ap.add_argument("--ref-cols", type=int, default=2048, help="weight rows per case in the reference arm's sample")
+    ap.add_argument("--tables", default=None, metavar="PATH", help="also write the long per-case tables (JSON) to this file")
+    ap.add_argument("--ref-cols", type=int, default=ORACLE_SAMPLE_ROWS, help="weight rows per case in the reference arm's sample")
     ap.add_argument("--case", default=None, metavar="M,N,K | M,H",
                     help="M,H: a few det_rmsnorm launches.  M,N,K: run only this shape: --steps eager det_linear_run calls over rotating weight copies "
                          "(a small, profiler-friendly workload; prints its own one-line JSON)")

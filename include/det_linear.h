@@ -56,7 +56,7 @@ typedef enum {
 } det_status_t;
 
 /* Storage format of the weight matrix.  Every format widens exactly to FP32 in registers (Eq. 2's
- * up()); the reduction order does not depend on it.  The paper's kernels take "16-bit weights" and
+ * up()); the reduction order does not depend on it.  The paper's kernels take 16-bit weights and
  * its seeded probe covers BF16 and FP32 weights. */
 typedef enum {
     DET_WEIGHT_BF16 = 0,            /* bfloat16 bit patterns, 2 bytes per element (default)        */
@@ -78,8 +78,8 @@ typedef struct {
 } det_linear_params_t;
 
 /*
- * Shape -> order parameters (rule R2: "compile-time constants selected by a pure function of the
- * problem shape"; R3: the split is shape-pure; R4: decode parameters never read M).  Pure host
+ * Shape -> order parameters (rule R2: the configuration is a constant chosen by the shape alone;
+ * R3: the split is shape-pure; R4: decode parameters never read M).  Pure host
  * function: touches no device, allocates nothing.  M, N, K >= 1 and each < 2^31, M*N < 2^40.
  * The `kernel` field reports the kernel for 16-byte aligned buffers.
  */

@@ -3,8 +3,8 @@
  * arithmetic: the hooks select among kernels and launch geometries that must all produce the same
  * bits (tile sizes, warp counts, pipeline depth and grid size are numerically inert: supplement C
  * on rule R2), and create streams restricted to a subset of the SMs so that tests can check that
- * the output does not depend on the SM count (rule R3: "independent of the device, its SM count,
- * and grid scheduling").  The paper has no counterpart for these functions.
+ * the output does not depend on the SM count (rule R3: the result may depend on neither the device,
+ * the number of SMs nor the way the grid is scheduled).  The paper has no counterpart for these functions.
  */
 #ifndef DET_LINEAR_TEST_H
 #define DET_LINEAR_TEST_H
@@ -50,7 +50,7 @@ DET_API det_status_t det_test_measure_fma_peak(int packed, double* tflops_out);
 DET_API det_status_t det_test_measure_read_bandwidth(const void* buf, size_t bytes, double* gbs_out);
 
 /*
- * Negative control for rule R3 (the paper's split-K ablation "none / ordered / atomic"): the decode
+ * Negative control for rule R3 (the paper's split-K ablation in supplement C: no split, ordered combine, atomic combine): the decode
  * order's segment partials for a requested split S_req (segments of whole 256-element blocks, as in
  * the library), combined with atomicAdd onto y (pre-set to the bias, or zero) in arrival order --
  * the scheme the rule forbids.  The output is close to det_linear_run's but its bits depend on grid

@@ -10,7 +10,7 @@ namespace detlin {
 
 constexpr int kOrderVersion = 1;
 constexpr int kSegmentGranule = 256;   // segment boundaries are multiples of this many k elements
-constexpr int kDecodeMaxM = 64;        // decode bucket edge (rule R2: "decode-shaped GEMMs (M <= 64)")
+constexpr int kDecodeMaxM = 64;        // decode bucket edge: rule R2 puts batches of up to 64 rows in the decode bucket
 
 enum KernelId : int { kKernelGeneric = 0, kKernelDecode = 1, kKernelPrefill = 2 };
 

@@ -59,8 +59,16 @@ extern "C" det_status_t det_linear_run_noalloc(int64_t M, int64_t N, int64_t K, 
                   p.S, (unsigned long long)(need * 4), (unsigned long long)(kNoallocScratchFloats * 4));
         return DET_ERR_UNSUPPORTED_SHAPE;
     }
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) { set_error("run_noalloc: device query: %s", cudaGetErrorString(e)); return DET_ERR_CUDA; }
+    if (major != 10) {
+        set_error("run_noalloc: device %d is sm_%dx; this library is built for sm_100a only (no fallback)", dev, major);
+        return DET_ERR_ARCH;
+    }
     float* scratch = nullptr;
-    cudaError_t e = scratch_address(&scratch);
+    e = scratch_address(&scratch);
     if (e != cudaSuccess) {
         set_error("run_noalloc: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
         return DET_ERR_CUDA;

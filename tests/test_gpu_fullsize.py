@@ -28,7 +28,7 @@ def sample_points(M, N, rng, count=1500):
 
 
 @pytest.mark.parametrize("name,K,N", inputs.LLAMA3_8B_LAYER)
-@pytest.mark.parametrize("M", [1, 8, 32])
+@pytest.mark.parametrize("M", inputs.DECODE_MS)
 def test_decode_full_size_sampled(name, K, N, M):
     x, W, b = inputs.make_case(M, N, K)
     got = run_gpu(x, W, b)
@@ -39,7 +39,7 @@ def test_decode_full_size_sampled(name, K, N, M):
 
 
 @pytest.mark.parametrize("name,K,N", inputs.PREFILL_SHAPES)
-@pytest.mark.parametrize("M", [128, 2048])
+@pytest.mark.parametrize("M", inputs.PREFILL_MS)
 def test_prefill_full_size_sampled(name, K, N, M):
     x, W, b = inputs.make_case(M, N, K)
     got = run_gpu(x, W, b)

@@ -97,6 +97,44 @@ def test_bench_reference_arm_runs_on_cpu():
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
 
 
+def test_bench_headline_is_the_short_last_line(tmp_path):
+    """The last line of stdout must be a short, self-contained JSON headline (a reader that keeps only a
+    few KB of the tail still gets value, roofline, cpu_baseline and e2e); the long tables go elsewhere."""
+    import io
+    sys.path.insert(0, ROOT)
+    import bench
+    line = {"metric": bench.METRIC, "value": 3000.12, "unit": bench.UNIT, "n_gpus": 1, "steps": 20, "warmup": 3,
+            "ms_per_step": 0.7, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": {"workload": "w" * 200, "l2": "x" * 60, "multi_gpu": "replicas only"},
+            "pct_of_hbm_peak": 45.0, "tflops_fp32": 34.0,
+            "clocks": {"sm_mhz": 1965.0, "sm_max_mhz": 1965.0, "samples": 12, "reasons": [], "window": "y" * 50},
+            "e2e": {"value": 2500.0, "unit": bench.UNIT, "h2d_bytes_per_step": 1, "d2h_bytes_per_step": 2},
+            "gpu_launches": 400,
+            "roofline": {"bound": "hbm", "achieved": 3000.0, "peak": 6543.1, "unit": "GB/s", "frac": 0.45, "traffic": 1,
+                         "algorithmic_bytes_per_launch": 1, "frac_of_binding_roof": 0.7, "peak_source": "m", "kernel": "k" * 90},
+            "cpu_baseline": {"value": 0.7, "unit": bench.UNIT, "cores": 16, "kind": "oracle", "sample": "s" * 90},
+            "decode_pct_of_binding_roof": {f"M{m}": [80.0] * 4 for m in (1, 4, 8, 16, 32)},
+            "prefill_pct_fp32_peak": [70.0] * 6, "lm_head_pct_of_binding_roof": [90.0] * 3, "stack_pct_hbm": [80.0, 60.0]}
+    tables = {"per_case": [{"name": "n", "us": 1.0}] * 2000}          # far larger than any tail window
+    out, err = io.StringIO(), io.StringIO()
+    path = tmp_path / "sub" / "tables.json"
+    bench.emit(line, tables, str(path), out=out, err=err)
+    last = out.getvalue().strip().splitlines()[-1]
+    assert len(last) < bench.HEADLINE_MAX_BYTES
+    got = json.loads(last)
+    for key in ("metric", "value", "unit", "n_gpus", "ms_per_step", "roofline", "cpu_baseline", "e2e", "clocks", "config"):
+        assert key in got
+    assert "per_case" not in got and len(out.getvalue()) < 2 * bench.HEADLINE_MAX_BYTES
+    assert json.loads(path.read_text())["tables"]["per_case"][0]["name"] == "n"
+    assert json.loads(err.getvalue())["headline"]["value"] == 3000.12
+    # an over-long headline sheds its optional digests instead of growing past the limit
+    line["config"]["workload"] = "w" * 700
+    out2 = io.StringIO()
+    bench.emit(line, {}, None, out=out2, err=io.StringIO())
+    got2 = json.loads(out2.getvalue().strip().splitlines()[-1])
+    assert len(out2.getvalue()) < bench.HEADLINE_MAX_BYTES + 2 and "roofline" in got2 and "stack_pct_hbm" not in got2
+
+
 _GLOO_WORKER = r"""
 import os, sys
 sys.path.insert(0, {root!r})

@@ -9,7 +9,7 @@ import torch
 
 from paper_2609_25624_b200 import binding as B
 from paper_2609_25624_b200 import inputs
-from tests.gpu_util import assert_bits_equal, run_gpu
+from tests.gpu_util import assert_bits_equal, oracle_y, run_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -22,12 +22,27 @@ CASES = [(1, 1024, 512), (8, 4096, 1024), (5, 300, 1001), (130, 200, 4096)]
 def test_noalloc_matches_planned_run_twice_in_a_row(M, N, K):
     x, W, b = inputs.make_case(M, N, K)
     want = run_gpu(x, W, b)                     # existing entry point: det_linear_plan + det_linear_run
+    assert_bits_equal(want, oracle_y(x, W, b), "planned run vs oracle")
     xd, Wd, bd = x.cuda(), W.cuda(), b.cuda()
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    B.det_linear_run_noalloc(xd, Wd, bd, y)     # first call on the device: resolves the scratch address
+    torch.cuda.synchronize()
     for call in range(2):
-        y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        y.fill_(float("nan"))
         B.det_linear_run_noalloc(xd, Wd, bd, y)
         torch.cuda.synchronize()
         assert_bits_equal(y.cpu().numpy(), want, f"call {call}")
+    # the entry point allocates nothing: the device's free memory does not shrink across calls (device-wide
+    # figure, so allow for another process allocating at the same moment by looking more than once)
+    for attempt in range(3):
+        free_before = torch.cuda.mem_get_info()[0]
+        for _ in range(4):
+            B.det_linear_run_noalloc(xd, Wd, bd, y)
+        torch.cuda.synchronize()
+        if torch.cuda.mem_get_info()[0] >= free_before:
+            break
+    else:
+        raise AssertionError("free device memory shrank across det_linear_run_noalloc calls")
     # a different problem in between must not disturb the next call (shared scratch, stale contents)
     x2, W2, b2 = inputs.make_case(3, 512, 768, seed=5)
     y2 = torch.empty(3, 512, dtype=torch.float32, device="cuda")
