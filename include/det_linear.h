@@ -9,11 +9,12 @@
  * of y do not depend on the SM count, the grid, the stream, co-scheduled work or, inside the
  * decode bucket (M <= 64), on M.
  *
- * Reduction order, version 1 (what "the same bits" means):
+ * Reduction order, version 2 (what "the same bits" means):
  *   bucket   = decode if M <= 64, else prefill                                  (R2, R4)
  *   decode : V = 4, L = 32, P = 1        prefill: V = 1, L = 1, P = 1 (strictly ascending k)
  *   K is cut into S contiguous segments of seg_len elements (a multiple of 256; only the last
- *   may be short); S is shape-pure and, for decode, independent of M               (R3, R4)
+ *   may be short); S is shape-pure and, for decode, independent of M: 2 segments for weight
+ *   matrices below 16384 rows (1 if K <= 256), no split above                      (R3, R4)
  *   inside a segment, chunks of V*L elements are walked in ascending k; "lane" l owns the V
  *   consecutive elements c + l*V + j; element j is accumulated with one fmaf into the lane's
  *   sub-chain j mod P, starting from +0.0f; elements beyond the segment end are skipped;
@@ -71,10 +72,10 @@ typedef struct {
     int32_t V, L, P;         /* order family parameters (see the header comment)                    */
     int64_t seg_len;         /* K elements per segment                                              */
     int32_t S;               /* number of segments, = ceil(K / seg_len)                             */
-    int32_t order_version;   /* version of the order definition, 1                                  */
+    int32_t order_version;   /* version of the order definition, 2                                  */
     int32_t kernel;          /* 0 generic, 1 decode (TMA pipeline), 2 prefill tile kernel           */
     int32_t weight_format;   /* det_weight_format_t of the plan (0 = BF16 for det_linear_plan_params)    */
-    uint64_t workspace_bytes;/* split-K partials: 4*S*M*N bytes when S > 1, else 0                  */
+    uint64_t workspace_bytes;/* split-K partials of the prefill bucket: 4*S*M*N bytes when S > 1; decode: 0 */
 } det_linear_params_t;
 
 /*
@@ -86,8 +87,10 @@ typedef struct {
 DET_API det_status_t det_linear_plan_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* out);
 
 /*
- * Create a plan for y[M,N] = x[M,K] * up(W[N,K])^T (+ b[N]) on the current device.  Allocates the
- * split-K partials workspace (device) when S > 1.  Returns NULL on failure (det_last_error()).
+ * Create a plan for y[M,N] = x[M,K] * up(W[N,K])^T (+ b[N]) on the current device.  Allocates a
+ * status word and, in the prefill bucket when S > 1, the split-K partials workspace (device); the
+ * decode bucket folds its segments inside the kernel and needs none.  Returns NULL on failure
+ * (det_last_error(), det_last_status()).
  * A plan may be used from one stream at a time: its workspace is not re-entrant; make one plan
  * per stream for concurrent use.  Destroy with det_linear_plan_destroy.
  */
@@ -119,14 +122,19 @@ DET_API det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K
 
 /*
  * Enqueue the computation on `stream` (a cudaStream_t; NULL = the legacy default stream) and
- * return without synchronising.  Eq. 2 with the order above; split-K partials, if any, are
- * combined by a second fixed-order pass (R3), never by atomics.
+ * return without synchronising.  Eq. 2 with the order above; the segment sums are folded in
+ * ascending order (R3) -- inside the kernel in the decode bucket, by a second fixed-order pass in the
+ * prefill bucket -- never by atomics.
  *   x : device, FP32, [M,K] row-major (row pitch K)
  *   W : device, BF16 bit patterns, [N,K] row-major (row pitch K): one weight row per output column
  *   b : device, FP32, [N], or NULL for no bias (then no final add happens at all)
  *   y : device, FP32, [M,N] row-major; overwritten; must not overlap the inputs
  * Buffers stay owned by the caller and must stay valid until the stream reaches the end of the
- * work.  The fast kernels need K % 8 == 0 and 16-byte aligned x, W, y; anything else runs a
+ * work.  W and b are parameters: they must be complete before the kernel that precedes this call in
+ * the stream STARTS (the decode kernel is launched with programmatic dependent launch and requests
+ * its first weight tiles, and reads b, before it waits for that kernel to finish; only x and y are
+ * touched after the wait).  If W or b were just written on the same stream -- a dequantise or copy
+ * kernel, a device-side random fill -- put another kernel or a synchronisation in between.  The fast kernels need K % 8 == 0 and 16-byte aligned x, W, y; anything else runs a
  * slower generic kernel that produces the same bits.  Errors: DET_ERR_INVALID_ARG for NULL
  * arguments, DET_ERR_CUDA if a launch fails.  Nothing is launched when an error is returned.
  */
@@ -228,8 +236,8 @@ DET_API det_status_t det_rmsnorm(const float* x, const float* g, float eps, int6
  * plan.  Inputs and output are passed as for det_linear_run (device pointers, same layouts, b may
  * be NULL); the result has the same bits.
  *
- * The split-K partials (needed only when the shape splits K, i.e. S > 1: 4*S*M*N bytes) live in a
- * 4 MiB array built into the library image, present on every GPU that loads the library until the
+ * The split-K partials (needed only in the prefill bucket, M > 64, when the shape splits K, i.e.
+ * S > 1: 4*S*M*N bytes) live in a 4 MiB array built into the library image, present on every GPU that loads the library until the
  * process exits.  A shape that needs more is rejected with DET_ERR_UNSUPPORTED_SHAPE and a message
  * that names both sizes; nothing is launched then.  All calls share that one array and it keeps the
  * last call's contents (nothing in it needs clearing: each call overwrites what it reads), so two
@@ -237,7 +245,8 @@ DET_API det_status_t det_rmsnorm(const float* x, const float* g, float eps, int6
  * issue them on one stream or order them yourself.
  *
  * The first call on each device looks up the array's device address (with that device current);
- * make that first call before starting any stream capture.  The kernels are the library's generic
+ * make that first call before starting any stream capture.  The address is kept for the life of the
+ * process: after a cudaDeviceReset the library must be reloaded before this entry point is used again.  The kernels are the library's generic
  * ones (any shape and alignment, not tuned for speed).  Enqueues on `stream`, no synchronisation.
  */
 DET_API det_status_t det_linear_run_noalloc(int64_t M, int64_t N, int64_t K, const float* x, const uint16_t* W,
@@ -246,7 +255,12 @@ DET_API det_status_t det_linear_run_noalloc(int64_t M, int64_t N, int64_t K, con
 /* Message of the last error on the calling thread ("" if none).  Never NULL. */
 DET_API const char* det_last_error(void);
 
-/* Version of the reduction-order definition implemented by this library (currently 1). */
+/* Status behind the last det_linear_plan* call of the calling thread: DET_OK if it returned a plan,
+ * otherwise why it returned NULL (DET_ERR_INVALID_ARG, DET_ERR_UNSUPPORTED_SHAPE, DET_ERR_ARCH,
+ * DET_ERR_ALLOC, DET_ERR_CUDA). */
+DET_API det_status_t det_last_status(void);
+
+/* Version of the reduction-order definition implemented by this library (currently 2). */
 DET_API int det_order_version(void);
 
 #ifdef __cplusplus

@@ -28,6 +28,24 @@ DET_API det_status_t det_test_plan_set_max_blocks(det_linear_plan_t* plan, int m
 DET_API det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant);
 
 /*
+ * Host-side fault injection: make the nth device allocation the library attempts from now on (1 = the
+ * next one) fail once with an out-of-memory error, without touching the device; 0 switches the hook
+ * off.  det_linear_plan* must then return NULL with det_last_status() == DET_ERR_ALLOC and free
+ * whatever it had already allocated.  Process-wide, not thread-safe: tests only.
+ */
+DET_API void det_test_fail_next_alloc(int nth);
+
+/*
+ * Bound of one device-side wait for the kernels launched through this plan (default 2 s), and flags:
+ * bit 0 (value 1) is a deliberate stall: thread block 0 of the decode kernel never
+ * requests the activations of its first stage, so the wait for that stage runs into the bound.  The
+ * kernel then records the timeout in the plan's status word, drains and returns (no trap, no endless
+ * loop; the other blocks finish normally), and det_linear_plan_check reports DET_ERR_DEVICE_TIMEOUT.
+ * The output of such a run is undefined.  Reset with (2000000000, 0).
+ */
+DET_API det_status_t det_test_plan_set_wait(det_linear_plan_t* plan, uint64_t wait_limit_ns, int flags);
+
+/*
  * Create a CUDA green context holding (at least) `sm_count` SMs of the current device and a
  * stream on it.  *stream_out receives a cudaStream_t usable with det_linear_run; *handle_out an
  * opaque handle for det_test_green_stream_destroy; *sm_granted the number of SMs in the

@@ -16,12 +16,14 @@ import numpy as np
 
 from . import build_oracle
 
-ORDER_VERSION = 1
+ORDER_VERSION = 2
 
 #: segment boundaries fall on multiples of this many k elements in both buckets
 SEGMENT_GRANULE = 256
-#: decode bucket edge (R2/R4: "decode-shaped GEMMs (M <= 64)")
+#: decode bucket edge (R2/R4: batches of up to 64 rows are decode-shaped)
 DECODE_MAX_M = 64
+#: decode bucket: weight matrices with at least this many rows are not split (they fill the machine)
+DECODE_NO_SPLIT_ROWS = 16384
 
 
 def _ceil_div(a: int, b: int) -> int:
@@ -39,18 +41,15 @@ def _segments_for(K: int, s_req: int):
 def split_request(M: int, N: int, K: int) -> int:
     """Requested number of K segments before clamping to what K allows.
 
-    Decode (never reads M, rule R4): 1 when N >= 4096 (enough rows to fill the machine, like the
-    paper's lm_head "prefers no split"); otherwise the smallest power of two with N*S >= 4096.
+    Decode (never reads M, rule R4): 1 when N >= 16384 (enough weight rows to keep every SM busy on its
+    own; the paper's lm_head likewise takes no split), otherwise 2.
     Prefill: the request in 1..16 that minimises rounds * (seg_len + overhead) * occupancy_factor,
     with tiles = number of 128x128 output tiles, units = tiles * S, rounds = ceil(units / 148),
     overhead = 8 k-steps per work unit plus 32 when partials are written and combined,
     occupancy_factor = 9 if units <= 148 else 8; ties go to the larger request.  The constants are
     frozen parts of the order definition (tuned once on a 148-SM part, never read from the device)."""
     if M <= DECODE_MAX_M:
-        s = 1
-        while N * s < 4096:
-            s *= 2
-        return s
+        return 1 if N >= DECODE_NO_SPLIT_ROWS else 2
     tiles = _ceil_div(M, 128) * _ceil_div(N, 128)
     best, best_cost = 1, None
     for s_req in range(1, 17):

@@ -80,6 +80,11 @@ def lib() -> ctypes.CDLL:
         L.det_rmsnorm.restype = i32
         L.det_last_error.restype = ctypes.c_char_p
         L.det_order_version.restype = i32
+        L.det_last_status.restype = i32
+        L.det_test_fail_next_alloc.argtypes = [i32]
+        L.det_test_fail_next_alloc.restype = None
+        L.det_test_plan_set_wait.argtypes = [p, ctypes.c_uint64, i32]
+        L.det_test_plan_set_wait.restype = i32
         L.det_test_plan_force_kernel.argtypes = [p, i32]
         L.det_test_plan_force_kernel.restype = i32
         L.det_test_plan_set_max_blocks.argtypes = [p, i32]
@@ -115,6 +120,11 @@ def det_last_error() -> str:
 
 def det_order_version() -> int:
     return int(lib().det_order_version())
+
+
+def det_last_status() -> int:
+    """Status behind the last det_linear_plan* call of this thread (DET_OK if it returned a plan)."""
+    return int(lib().det_last_status())
 
 
 def det_linear_plan_params(M: int, N: int, K: int) -> Params:
@@ -153,7 +163,7 @@ class Plan:
         else:
             self._h = lib().det_linear_plan_w(self.M, self.N, self.K, self.wfmt)
         if not self._h:
-            raise DetLinearError(-1, det_last_error())
+            raise DetLinearError(det_last_status(), det_last_error())
 
     def close(self):
         if getattr(self, "_h", None):
@@ -329,6 +339,17 @@ def det_test_plan_set_max_blocks(plan: Plan, max_blocks: int) -> None:
 
 def det_test_plan_set_variant(plan: Plan, variant: int) -> None:
     _check(lib().det_test_plan_set_variant(plan.handle, variant))
+
+
+def det_test_fail_next_alloc(nth: int = 1) -> None:
+    """Host-side fault injection: the nth device allocation from now on fails once (0 = off)."""
+    lib().det_test_fail_next_alloc(int(nth))
+
+
+def det_test_plan_set_wait(plan: Plan, wait_limit_ns: int, withhold_first_copy: bool = False) -> None:
+    """Bound of one device-side wait for this plan's kernels; optionally stall one wait on purpose."""
+    flags = 1 if withhold_first_copy else 0
+    _check(lib().det_test_plan_set_wait(plan.handle, int(wait_limit_ns), flags))
 
 
 def det_test_green_stream_create(sm_count: int):

@@ -36,6 +36,7 @@ def _stale(target, deps):
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile what is out of date and link the shared library; return its path."""
     nvcc = os.environ.get("NVCC", "nvcc")
+    extra = os.environ.get("DET_EXTRA_NVCC_FLAGS", "").split()      # e.g. instrumentation defines for experiments
     os.makedirs(OBJ_DIR, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers += [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE) if f.endswith(".h")]
@@ -46,7 +47,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         op = os.path.join(OBJ_DIR, os.path.splitext(src)[0] + tag + ".o")
         objs.append(op)
         if force or _stale(op, [sp] + headers):
-            cmd = [nvcc, *NVCC_FLAGS, *defines, "-x", "cu", "-c", sp, "-o", op]
+            cmd = [nvcc, *NVCC_FLAGS, *extra, *defines, "-x", "cu", "-c", sp, "-o", op]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))

@@ -9,6 +9,7 @@
 namespace detlin {
 
 static thread_local char g_err[512] = "";
+static thread_local int g_last_status = DET_OK;   // status behind a NULL plan (det_last_status)
 
 void set_error(const char* fmt, ...)
 {
@@ -56,6 +57,15 @@ static bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, 
     return true;
 }
 
+// Device allocation with the test hook of det_test_fail_next_alloc: the next `skip`-th call fails once
+// with cudaErrorMemoryAllocation without touching the device.
+static int g_fail_alloc_countdown = 0;          // 0 = off; n = the n-th allocation from now fails
+static cudaError_t device_alloc(void** p, size_t bytes)
+{
+    if (g_fail_alloc_countdown > 0 && --g_fail_alloc_countdown == 0) { *p = nullptr; return cudaErrorMemoryAllocation; }
+    return cudaMalloc(p, bytes);
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static det_status_t run_device(det_linear_plan_t* plan, const float* x, const void* W, const float* b, float* y,
@@ -85,26 +95,33 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const vo
     const bool fast_ok = (p.K % k_align == 0) && (p.K % 4 == 0) && p.K <= (1 << 30) && p.N <= (1 << 30) && aligned16(x) && aligned16(W) && aligned16(y);
     if (!fast_ok) kernel = kKernelGeneric;
 
+    a.wait_limit_ns = plan->wait_limit_ns;
+    a.test_flags = plan->test_flags;
+
     cudaError_t e = cudaSuccess;
     if (kernel == kKernelDecode) {
-        DecodeConfig cfg;
-        if (!decode_config_for(p.M, plan->n_count, p.K, p.S, p.weight_format, plan->variant, &cfg)) {
-            set_error("run: no decode configuration for this shape/variant");
-            return DET_ERR_INVALID_ARG;
+        // the tiling is a function of the plan and the device: chosen once, then cached
+        if (plan->decode_cfg_variant != plan->variant) {
+            if (!decode_config_for(p.M, plan->n_count, p.K, p.S, p.weight_format, plan->variant, &plan->decode_cfg)) {
+                set_error("run: no decode configuration for this shape/variant");
+                return DET_ERR_INVALID_ARG;
+            }
+            plan->decode_cfg_variant = plan->variant;
         }
+        const DecodeConfig& cfg = plan->decode_cfg;
         if (plan->map_w_ptr != W || plan->map_x_ptr != x || plan->map_cfg_id != cfg.id + 1024 * p.weight_format) {
             const CUtensorMapDataType wdt = p.weight_format == DET_WEIGHT_FP32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                             : p.weight_format == DET_WEIGHT_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
                                                                                  : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
             if (!encode_2d(&plan->map_w, wdt, p.weight_format == DET_WEIGHT_FP32 ? 4 : 2, W, (uint64_t)plan->n_count, (uint64_t)p.K,
-                           (uint32_t)cfg.rt, (uint32_t)cfg.kc, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+                           (uint32_t)(cfg.rt * cfg.wr), (uint32_t)(cfg.kc < 256 ? cfg.kc : 256), CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
                 return DET_ERR_CUDA;
             if (!encode_2d(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, x, (uint64_t)p.M, (uint64_t)p.K,
-                           (uint32_t)(cfg.mt * cfg.wm), (uint32_t)cfg.kc, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+                           (uint32_t)(cfg.mt * cfg.wm), (uint32_t)(cfg.kc < 256 ? cfg.kc : 256), CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
                 return DET_ERR_CUDA;
             plan->map_w_ptr = W; plan->map_x_ptr = x; plan->map_cfg_id = cfg.id + 1024 * p.weight_format;
         }
-        e = launch_decode(a, &plan->map_w, &plan->map_x);
+        e = launch_decode(a, cfg, &plan->map_w, &plan->map_x);
     } else if (kernel == kKernelPrefill) {
         e = launch_prefill(a);
     } else {
@@ -136,29 +153,32 @@ det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K, int64_
                                          int32_t wfmt)
 {
     det_linear_params_t prm;
-    if (fill_params(M, N, K, &prm) != DET_OK) return nullptr;
+    g_last_status = fill_params(M, N, K, &prm);
+    if (g_last_status != DET_OK) return nullptr;
+    g_last_status = DET_ERR_INVALID_ARG;
     if (wfmt < DET_WEIGHT_BF16 || wfmt > DET_WEIGHT_FP32) { set_error("plan: unknown weight format %d", wfmt); return nullptr; }
     if (n_begin < 0 || n_count < 1 || n_begin > N - n_count || ldy < n_count) {
         set_error("plan: shard [%lld, %lld) with row pitch %lld does not fit a layer with N = %lld", (long long)n_begin,
                   (long long)(n_begin + n_count), (long long)ldy, (long long)N);
         return nullptr;
     }
-    prm.workspace_bytes = prm.S > 1 ? 4ull * (uint64_t)prm.S * (uint64_t)M * (uint64_t)n_count : 0;
+    prm.workspace_bytes = (prm.bucket == 1 && prm.S > 1) ? 4ull * (uint64_t)prm.S * (uint64_t)M * (uint64_t)n_count : 0;
     prm.weight_format = wfmt;
     if (wfmt == DET_WEIGHT_FP32) prm.kernel = (K % 4 == 0) ? (prm.bucket == 0 ? kKernelDecode : kKernelPrefill) : kKernelGeneric;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) { cuda_fail("cudaGetDevice", e); return nullptr; }
+    if (e != cudaSuccess) { g_last_status = cuda_fail("cudaGetDevice", e); return nullptr; }
     cudaDeviceProp prop;
     e = cudaGetDeviceProperties(&prop, dev);
-    if (e != cudaSuccess) { cuda_fail("cudaGetDeviceProperties", e); return nullptr; }
+    if (e != cudaSuccess) { g_last_status = cuda_fail("cudaGetDeviceProperties", e); return nullptr; }
     if (prop.major != 10) {
+        g_last_status = DET_ERR_ARCH;
         set_error("plan: device %d is sm_%d%d; this library is built for sm_100a only (no fallback)", dev, prop.major,
                   prop.minor);
         return nullptr;
     }
     det_linear_plan_t* plan = new (std::nothrow) det_linear_plan_t();
-    if (!plan) { set_error("plan: host allocation failed"); return nullptr; }
+    if (!plan) { g_last_status = DET_ERR_ALLOC; set_error("plan: host allocation failed"); return nullptr; }
     memset(plan, 0, sizeof *plan);
     plan->prm = prm;
     plan->n_begin = n_begin;
@@ -168,14 +188,18 @@ det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K, int64_
     plan->sm_count = prop.multiProcessorCount;
     plan->forced_kernel = -1;
     plan->map_cfg_id = -1;
-    e = cudaMalloc(&plan->status, sizeof(DeviceStatus));
+    plan->decode_cfg_variant = -1;
+    plan->wait_limit_ns = kDefaultWaitLimitNs;
+    g_last_status = DET_OK;
+    e = device_alloc(reinterpret_cast<void**>(&plan->status), sizeof(DeviceStatus));
     if (e == cudaSuccess) e = cudaMemset(plan->status, 0, sizeof(DeviceStatus));
-    if (e == cudaSuccess && prm.workspace_bytes) e = cudaMalloc(&plan->partials, prm.workspace_bytes);
+    if (e == cudaSuccess && prm.workspace_bytes) e = device_alloc(reinterpret_cast<void**>(&plan->partials), prm.workspace_bytes);
     if (e != cudaSuccess) {
-        set_error("plan: device allocation of %llu bytes failed: %s", (unsigned long long)prm.workspace_bytes,
-                  cudaGetErrorString(e));
+        g_last_status = DET_ERR_ALLOC;
+        set_error("plan: device allocation (status word, %llu bytes of split-K workspace) failed: %s",
+                  (unsigned long long)prm.workspace_bytes, cudaGetErrorString(e));
         cudaGetLastError();
-        det_linear_plan_destroy(plan);
+        det_linear_plan_destroy(plan);              // frees whatever was allocated before the failure
         return nullptr;
     }
     return plan;
@@ -214,9 +238,14 @@ static det_status_t run_host_impl(det_linear_plan_t* plan, const float* x_host, 
     const size_t xb = (size_t)p.M * p.K * 4, yb = (size_t)p.M * p.N * 4;
     cudaError_t e;
     if (!plan->x_stage) {
-        e = cudaMalloc(&plan->x_stage, xb);
-        if (e == cudaSuccess) e = cudaMalloc(&plan->y_stage, yb);
-        if (e != cudaSuccess) { set_error("run_host: staging allocation failed: %s", cudaGetErrorString(e)); cudaGetLastError(); return DET_ERR_ALLOC; }
+        e = device_alloc(reinterpret_cast<void**>(&plan->x_stage), xb);
+        if (e == cudaSuccess) e = device_alloc(reinterpret_cast<void**>(&plan->y_stage), yb);
+        if (e != cudaSuccess) {
+            set_error("run_host: staging allocation failed: %s", cudaGetErrorString(e));
+            cudaGetLastError();
+            if (plan->x_stage) { cudaFree(plan->x_stage); plan->x_stage = nullptr; }     // all or nothing: a later call retries both
+            return DET_ERR_ALLOC;
+        }
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     e = cudaMemcpyAsync(plan->x_stage, x_host, xb, cudaMemcpyHostToDevice, st);
@@ -349,8 +378,8 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
         DecodeConfig c;
         if (decode_config_for(p.M, plan->n_count, p.K, p.S, p.weight_format, plan->variant, &c))
             snprintf(tiling, sizeof tiling,
-                     "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"kc\": %d, \"stages\": %d, \"blocks_per_sm\": %d}", c.mt,
-                     c.wm, c.rt, c.wr, c.kc, c.stages, decode_config_occupancy(p.weight_format, c));
+                     "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"sk\": %d, \"kc\": %d, \"stages\": %d, \"blocks_per_sm\": %d}",
+                     c.mt, c.wm, c.rt, c.wr, c.sk, c.kc, c.stages, decode_config_occupancy(p.weight_format, c, p.S));
     }
     char ptile[64] = "null";
     if (p.kernel == kKernelPrefill) {
@@ -391,6 +420,8 @@ det_status_t det_argmax_rows(const float* y, int64_t M, int64_t N, int32_t* idx,
 
 const char* det_last_error(void) { return g_err; }
 
+det_status_t det_last_status(void) { return static_cast<det_status_t>(g_last_status); }
+
 int det_order_version(void) { return kOrderVersion; }
 
 // ---------------------------------------------------------------------------------------------
@@ -429,6 +460,19 @@ det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
         return DET_ERR_INVALID_ARG;
     }
     plan->variant = variant;
+    return DET_OK;
+}
+
+void det_test_fail_next_alloc(int nth)
+{
+    g_fail_alloc_countdown = nth > 0 ? nth : 0;
+}
+
+det_status_t det_test_plan_set_wait(det_linear_plan_t* plan, uint64_t wait_limit_ns, int flags)
+{
+    if (!plan || wait_limit_ns == 0 || flags < 0 || flags > 1) { set_error("set_wait: bad argument"); return DET_ERR_INVALID_ARG; }
+    plan->wait_limit_ns = wait_limit_ns;
+    plan->test_flags = flags;
     return DET_OK;
 }
 

@@ -8,8 +8,11 @@
 
 namespace detlin {
 
-constexpr int kOrderVersion = 1;
+constexpr int kOrderVersion = 2;
 constexpr int kSegmentGranule = 256;   // segment boundaries are multiples of this many k elements
+constexpr int64_t kDecodeNoSplitRows = 16384;   // decode bucket: weight matrices with at least this many rows are not split
+constexpr int kDecodeMaxSegments = 8;  // most K segments the decode kernel folds inside a thread block
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;   // bound of one device-side wait: 2 s
 constexpr int kDecodeMaxM = 64;        // decode bucket edge: rule R2 puts batches of up to 64 rows in the decode bucket
 
 enum KernelId : int { kKernelGeneric = 0, kKernelDecode = 1, kKernelPrefill = 2 };
@@ -42,12 +45,14 @@ struct LaunchArgs {
     int sm_count;
     int max_blocks;       // 0 = automatic
     int variant;          // 0 = automatic
+    unsigned long long wait_limit_ns;   // bound of one device-side wait (decode kernel)
+    int test_flags;       // decode kernel test hooks (0 outside the tests)
 };
 
 cudaError_t launch_generic(const LaunchArgs& a, int bucket);
 // Second pass of split-K: y[m,n] = (((P0 + P1) + P2) + ...) (+ b[n]); rule R3.
 cudaError_t launch_combine(const LaunchArgs& a);
-cudaError_t launch_decode(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x);
+
 cudaError_t launch_prefill(const LaunchArgs& a);
 // rows per thread (tile height = 16 x this) the prefill kernel uses for batch size M; schedule only
 int prefill_rows_per_thread(int64_t M);
@@ -60,14 +65,15 @@ cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cu
 // Decode-kernel tiling chosen for a shape (numerically inert); used by the host to build the
 // tensor maps with matching box sizes.
 struct DecodeConfig {
-    int mt, wm, rt, wr, kc, stages;   // warp tile (mt x rt), warps (wm x wr), k per stage, ring depth
+    int mt, wm, rt, wr, sk, kc, stages;   // warp tile (mt x rt), warps (wm x wr) x sk segment groups, k per stage, ring depth
     int id;
 };
 // S = number of K segments of the order (it only scales the unit count in the schedule's cost model)
 bool decode_config_for(int64_t M, int64_t N, int64_t K, int S, int wfmt, int variant, DecodeConfig* out);
 int decode_num_variants();
-// resident blocks per SM of a tiling on the current device (schedule information only)
-int decode_config_occupancy(int wfmt, const DecodeConfig& cfg);
+cudaError_t launch_decode(const LaunchArgs& a, const DecodeConfig& cfg, const CUtensorMap* map_w, const CUtensorMap* map_x);
+// resident blocks per SM of a tiling on the current device for an order with S segments (schedule information only)
+int decode_config_occupancy(int wfmt, const DecodeConfig& cfg, int S);
 
 }  // namespace detlin
 
@@ -83,6 +89,11 @@ struct det_linear_plan {
     int forced_kernel;               // -1 automatic
     int max_blocks;
     int variant;
+    unsigned long long wait_limit_ns;
+    int test_flags;
+    // the decode tiling chosen for this plan (schedule only; cached so that a run does no search)
+    detlin::DecodeConfig decode_cfg;
+    int decode_cfg_variant;          // variant the cached tiling was chosen for, -1 = none yet
     // tensor-map cache for the decode kernel (keyed by the pointers they were built for)
     const void* map_w_ptr;
     const void* map_x_ptr;

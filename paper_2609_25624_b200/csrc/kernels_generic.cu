@@ -7,38 +7,38 @@
 
 namespace detlin {
 
-// Decode order (V=4, L=32, P=1): one warp per (row n, segment s); lane l owns k = c + 4l + j in every
-// 128-element chunk and accumulates them in ascending order into one chain; the 32 lanes are summed
-// adjacent-first.
+// Decode order (V=4, L=32, P=1, S segments): one warp per weight row n.  Lane l owns k = c + 4l + j in
+// every 128-element chunk of a segment and accumulates them in ascending order into one chain; the 32
+// lanes are summed adjacent-first; the warp walks the S segments in ascending order and folds their sums
+// as it goes (rule R3), so this bucket needs no workspace and no second pass.
 template <int WF>
 __global__ void __launch_bounds__(256)
 generic_decode_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type* __restrict__ W, const float* __restrict__ b,
-                      float* __restrict__ out, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int direct, int64_t ldy)
+                      float* __restrict__ y, int64_t M, int64_t N, int64_t K, int64_t seg_len, int S, int64_t ldy)
 {
     const int lane = threadIdx.x & 31;
-    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (warp >= N * S) return;
-    const int64_t n = warp / S;
-    const int s = (int)(warp % S);
-    const int64_t k_lo = (int64_t)s * seg_len;
-    const int64_t k_hi = (k_lo + seg_len < K) ? k_lo + seg_len : K;
+    const int64_t n = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (n >= N) return;
     const typename WeightElem<WF>::type* wrow = W + n * K;
     for (int64_t m = 0; m < M; ++m) {
         const float* xrow = x + m * K;
-        float a = 0.0f;
-        for (int64_t c = k_lo; c < k_hi; c += 128) {
-            const int64_t k0 = c + 4 * lane;
+        float t = 0.0f;
+        for (int s = 0; s < S; ++s) {
+            const int64_t k_lo = (int64_t)s * seg_len;
+            const int64_t k_hi = (k_lo + seg_len < K) ? k_lo + seg_len : K;
+            float a = 0.0f;
+            for (int64_t c = k_lo; c < k_hi; c += 128) {
+                const int64_t k0 = c + 4 * lane;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int64_t k = k0 + j;
-                if (k < k_hi) a = __fmaf_rn(xrow[k], up_elem<WF>(wrow[k]), a);
+                for (int j = 0; j < 4; ++j) {
+                    const int64_t k = k0 + j;
+                    if (k < k_hi) a = __fmaf_rn(xrow[k], up_elem<WF>(wrow[k]), a);
+                }
             }
+            const float p = lane_tree_sum(a);
+            t = (s == 0) ? p : __fadd_rn(t, p);
         }
-        const float t = lane_tree_sum(a);
-        if (lane == 0) {
-            if (direct) out[m * ldy + n] = b ? __fadd_rn(t, b[n]) : t;
-            else        out[((int64_t)s * M + m) * N + n] = t;
-        }
+        if (lane == 0) y[m * ldy + n] = b ? __fadd_rn(t, b[n]) : t;
     }
 }
 
@@ -85,13 +85,14 @@ static cudaError_t launch_generic_t(const LaunchArgs& a, int bucket)
 {
     typedef typename WeightElem<WF>::type WT;
     const WT* W = static_cast<const WT*>(a.W);
+    if (bucket == 0) {
+        const int64_t blocks = (a.N + 7) / 8;
+        generic_decode_kernel<WF><<<(unsigned)blocks, 256, 0, a.stream>>>(a.x, W, a.b, a.y, a.M, a.N, a.K, a.seg_len, a.S, a.ldy);
+        return cudaGetLastError();
+    }
     const int direct = (a.S == 1);
     float* out = direct ? a.y : a.partials;
-    if (bucket == 0) {
-        const int64_t warps = a.N * a.S;
-        const int64_t blocks = (warps + 7) / 8;
-        generic_decode_kernel<WF><<<(unsigned)blocks, 256, 0, a.stream>>>(a.x, W, a.b, out, a.M, a.N, a.K, a.seg_len, a.S, direct, a.ldy);
-    } else {
+    {
         // grid.y carries M (< 65536 per launch); larger M is cut into slabs of rows
         const int64_t max_y = 32768;
         for (int64_t m0 = 0; m0 < a.M; m0 += max_y) {

@@ -52,7 +52,7 @@ extern "C" det_status_t det_linear_run_noalloc(int64_t M, int64_t N, int64_t K, 
     det_linear_params_t p;
     det_status_t st = fill_params(M, N, K, &p);
     if (st != DET_OK) return st;
-    const uint64_t need = p.S > 1 ? (uint64_t)p.S * (uint64_t)M * (uint64_t)N : 0;
+    const uint64_t need = p.workspace_bytes / 4;            // split-K partials of the prefill bucket, in floats
     if (need > kNoallocScratchFloats) {
         set_error("run_noalloc: this shape splits K into %d segments and needs %llu bytes of partials; the built-in "
                   "scratch holds %llu bytes (use det_linear_plan + det_linear_run for larger problems)",
@@ -76,7 +76,7 @@ extern "C" det_status_t det_linear_run_noalloc(int64_t M, int64_t N, int64_t K, 
     LaunchArgs a{};
     a.x = x; a.W = W; a.b = b; a.y = y;
     a.wfmt = DET_WEIGHT_BF16;
-    a.partials = p.S > 1 ? scratch : nullptr;    // every partial is written by the first pass before the
+    a.partials = need ? scratch : nullptr;       // every partial is written by the first pass before the
     a.M = M; a.N = N; a.K = K; a.ldy = N;                   // second pass reads it: nothing has to start at zero
     a.seg_len = p.seg_len; a.S = p.S;
     a.stream = static_cast<cudaStream_t>(stream);

@@ -18,23 +18,23 @@ static void segments_for(int64_t K, int64_t s_req, int64_t* seg_len, int64_t* S)
 }
 
 // Requested split factor before clamping to what K allows.
-//  decode : no split once N alone provides 4096 rows of parallel work (like the paper's lm_head,
-//           which "prefers no split"); below that the smallest power of two with N*S >= 4096.
-//           Never reads M (rule R4).
+//  decode : 1 when N >= 16384 (that many weight rows keep every SM busy on their own; the paper's
+//           lm_head likewise takes no split), otherwise 2: two segments let one thread block keep
+//           eight warps busy on a single 28-row weight tile -- 4096 rows over 148 SMs -- and fold
+//           the two segment sums inside the block, without a workspace or a second launch.  Never
+//           reads M (rule R4).  Measured on B200 before the freeze: against no split the small
+//           matrices gain up to 1.9x at batch 4 .. 8; four segments cost the large batches 5 %
+//           (one more lane tree per segment and output) and gain nothing further.
 //  prefill: the request in 1..16 that minimises  rounds * (seg_len + overhead) * occupancy_factor
 //           where tiles counts 128x128 output tiles, units = tiles * S, rounds = ceil(units / 148),
 //           overhead = 8 k-steps per work unit plus 32 when partials have to be written and combined,
 //           and occupancy_factor = 9 when units <= 148 (one block per SM) else 8; ties go to the
 //           larger split.  148 and the overheads were measured once on a B200 and are frozen
 //           constants of the order definition: the rule is a pure function of (M, N, K) and never
-//           reads the device (rule R2: "tuned once offline and pinned").
+//           reads the device (rule R2: configurations are tuned once, offline, and then pinned).
 static int split_request(int64_t M, int64_t N, int64_t K)
 {
-    if (M <= kDecodeMaxM) {
-        int s = 1;
-        while (N * s < 4096) s *= 2;
-        return s;
-    }
+    if (M <= kDecodeMaxM) return N >= kDecodeNoSplitRows ? 1 : 2;
     const int64_t tiles = ceil_div(M, 128) * ceil_div(N, 128);
     int best = 1;
     int64_t best_cost = -1;
@@ -72,7 +72,8 @@ det_status_t fill_params(int64_t M, int64_t N, int64_t K, det_linear_params_t* o
     p.order_version = kOrderVersion;
     p.weight_format = DET_WEIGHT_BF16;
     p.kernel = (K % 8 == 0) ? (p.bucket == 0 ? kKernelDecode : kKernelPrefill) : kKernelGeneric;
-    p.workspace_bytes = p.S > 1 ? (uint64_t)4 * (uint64_t)p.S * (uint64_t)M * (uint64_t)N : 0;
+    // the decode bucket folds its segments inside the kernels; the prefill bucket combines in a second pass
+    p.workspace_bytes = (p.bucket == 1 && p.S > 1) ? (uint64_t)4 * (uint64_t)p.S * (uint64_t)M * (uint64_t)N : 0;
     *out = p;
     return DET_OK;
 }

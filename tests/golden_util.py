@@ -13,9 +13,11 @@ def _f32_from_bits(b):
 
 def _parse_x(field):
     field = field.strip()
-    if field.startswith("K512:"):
-        x = [1.0] * 512
-        for item in field[len("K512:"):].split(","):
+    if field[:1] in ("K", "Z") and ":" in field and field[1:field.index(":")].isdigit():
+        # "K<n>: i=v, ..." = a row of n ones with the listed overrides; "Z<n>: ..." = a row of n zeros
+        n = int(field[1:field.index(":")])
+        x = [1.0 if field[0] == "K" else 0.0] * n
+        for item in field[field.index(":") + 1:].split(","):
             i, v = item.split("=")
             x[int(i)] = _parse_val(v.strip())
         return x

@@ -51,7 +51,8 @@ def test_decode_bit_exact_all_tilings(M, N, K):
             break
         assert_bits_equal(got, want, f"variant={variant}")
         n_tilings = variant
-    assert n_tilings >= 4
+    # tilings whose segment groups do not divide S cannot run the shape
+    assert n_tilings >= (4 if oracle.order_params(M, N, K)["S"] == 2 else 2)
     assert_bits_equal(run_gpu(x, W, b, max_blocks=1), want, "one block")
     assert_bits_equal(run_gpu(x, W, b, max_blocks=3), want, "three blocks")
 

@@ -53,16 +53,27 @@ def test_shards_reproduce_the_whole_layer(M, N, K, world):
 
 
 def test_shard_uses_the_layers_split_not_its_own():
-    """N = 1024 splits K in four (N * S >= 4096); a 256-column shard on its own would be planned with
-    S = 16 -> different bits.  The shard plan must keep the layer's S."""
-    M, N, K = 2, 1024, 4096
-    assert oracle.order_params(M, N, K)["S"] != oracle.order_params(M, 256, K)["S"]
+    """Prefill bucket: the layer (128, 4096, 4096) splits K in 8, a 1024-column shard planned on its own
+    would split it in 16 -> different bits.  The shard plan must keep the layer's S.  The same in the
+    decode bucket: a layer of 16384 rows is not split, a quarter of it planned on its own would be."""
+    M, N, K = 128, 4096, 4096
+    assert oracle.order_params(M, N, K)["S"] != oracle.order_params(M, N // 4, K)["S"]
+    x, W, b = inputs.make_case(M, N, K)
+    ns = np.arange(0, N, 37)
+    ms = (np.arange(len(ns)) * 5) % M
+    want = oracle.linear_sampled(x.numpy(), inputs.bf16_bits(W), b.numpy(), ms, ns)
+    got = run_sharded(x, W, b, 4, in_place=True)
+    assert_bits_equal(got[ms, ns], want, "layer order")
+    alone = run_gpu(x, W[:1024].contiguous(), b[:1024].contiguous())
+    assert not np.array_equal(alone.view(np.uint32), got[:, :1024].view(np.uint32))
+    # decode bucket
+    M, N, K = 2, 16384, 1024
+    assert oracle.order_params(M, N, K)["S"] != oracle.order_params(M, N // 4, K)["S"]
     x, W, b = inputs.make_case(M, N, K)
     want = oracle_y(x, W, b)
-    got = run_sharded(x, W, b, 4, in_place=True)
-    assert_bits_equal(got, want, "layer order")
-    alone = run_gpu(x, W[:256].contiguous(), b[:256].contiguous())
-    assert not np.array_equal(alone.view(np.uint32), want[:, :256].view(np.uint32))
+    assert_bits_equal(run_sharded(x, W, b, 4, in_place=True), want, "decode shards")
+    alone = run_gpu(x, W[:4096].contiguous(), b[:4096].contiguous())
+    assert not np.array_equal(alone.view(np.uint32), want[:, :4096].view(np.uint32))
 
 
 def test_shard_other_formats_and_no_bias():

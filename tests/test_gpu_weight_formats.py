@@ -48,7 +48,8 @@ def test_decode_bit_exact_all_tilings(M, N, K, wfmt):
             break
         assert_bits_equal(got, want, f"variant={variant}")
         n_tilings = variant
-    assert n_tilings >= 4
+    # tilings whose segment groups do not divide S cannot run the shape
+    assert n_tilings >= (4 if oracle.order_params(M, N, K)["S"] == 2 else 2)
     assert_bits_equal(run_gpu(x, W, b, max_blocks=3), want, "three blocks")
     assert_bits_equal(run_gpu(x, W, None), oracle_y(x, W, None), "no bias")
 

@@ -48,7 +48,7 @@ def test_plan_params_rule_and_oracle_agree(built_lib):
             for K in (1, 7, 8, 255, 256, 257, 512, 1000, 3072, 4096, 14336):
                 p = B.det_linear_plan_params(M, N, K)
                 assert p.as_dict() == oracle.order_params(M, N, K), (M, N, K)
-                assert p.workspace_bytes == (4 * p.S * M * N if p.S > 1 else 0)
+                assert p.workspace_bytes == (4 * p.S * M * N if (p.S > 1 and M > 64) else 0)   # decode folds in-kernel
                 assert p.kernel == (0 if K % 8 else (1 if M <= 64 else 2))
     # decode parameters never read M (rule R4)
     ref = B.det_linear_plan_params(1, 1024, 512).as_dict()
@@ -65,7 +65,7 @@ def test_bad_shapes_are_rejected_with_a_message(built_lib):
         assert B.det_last_error() != ""
     rc = B.lib().det_linear_plan_params(1, 1, 8, None)
     assert rc == 1
-    assert B.det_order_version() == 1
+    assert B.det_order_version() == 2
 
 
 def test_null_arguments_do_not_touch_the_device(built_lib):

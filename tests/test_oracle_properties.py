@@ -128,10 +128,10 @@ def test_order_params_rule():
             assert oracle.order_params(M, N, K) == ref
     # benchmark shapes
     assert oracle.order_params(1, 1024, 512) == dict(bucket="decode", V=4, L=32, P=1, seg_len=256, S=2,
-                                                     order_version=1)
+                                                     order_version=2)
     for (N, K) in [(4096, 4096), (6144, 4096), (28672, 4096), (4096, 14336), (128256, 4096)]:
         p = oracle.order_params(8, N, K)
-        assert (p["S"], p["seg_len"]) == (1, K)
+        assert (p["S"], p["seg_len"]) == ((1, K) if N >= 16384 else (2, K // 2))
     # every segment non-empty, boundaries on multiples of 256, all of K covered
     for M in (1, 64, 65, 128, 2048):
         for N in (1, 100, 1000, 4096, 28672):

@@ -13,8 +13,8 @@ from tests.gpu_util import assert_bits_equal, oracle_y, run_gpu
 
 pytestmark = pytest.mark.gpu
 
-# (M, N, K): split-K decode (S = 2, uses the scratch), decode without split, ragged K (generic path,
-# S = 4), prefill with split (S = 8, uses the scratch)
+# (M, N, K): decode with two segments, twice (folded inside the kernel: no scratch), ragged K,
+# prefill with split (S = 8: the partials go through the built-in scratch)
 CASES = [(1, 1024, 512), (8, 4096, 1024), (5, 300, 1001), (130, 200, 4096)]
 
 
