@@ -293,6 +293,174 @@ int det_oracle_rmsnorm(const float *x, const float *g, float eps, int64_t M, int
     return 0;
 }
 
+/*
+ * Fixed-order decode attention (an extension: the paper keeps vendor attention and names the reductions
+ * outside the linear layers -- "fixed-order attention" in particular -- as the residual channel of
+ * cross-run divergence).  One query row per (batch, head) attends to T cached keys and values:
+ *
+ *   q [B, Hq, D], k and v [B, Hkv, T, D] (Hq a multiple of Hkv; query head h reads KV head h / (Hq / Hkv)),
+ *   o [B, Hq, D], all binary32, row-major.
+ *
+ * Every step is one IEEE-754 binary32 operation, in an order fixed by (T, D) alone:
+ *   1. s_j = dot(q, k_j) * scale.  The dot product runs in the decode lane order over D: chunks of 128
+ *      ascending, "lane" l owns the 4 consecutive elements c + 4l + jj, one fmaf per element from +0.0f,
+ *      elements beyond D skipped, the 32 lane sums added by the adjacent-first tree; then one multiply.
+ *   2. m = max_j s_j (comparisons only: order-free).
+ *   3. e_j = exp_det(s_j - m): one subtraction, then det_oracle_exp below (its own fixed sequence).
+ *   4. l = sum_j e_j in the same lane order over j: chunks of 128 keys ascending, lane l owns keys
+ *      c + 4l + jj, one addition per key from +0.0f, keys beyond T skipped, adjacent-first lane tree.
+ *   5. for every d: the keys are cut into segments of 256 (the last may be short); inside a segment
+ *      a = fmaf(e_j, v_j[d], a) from +0.0f with j ascending; the segment sums are added left to right in
+ *      ascending segment order; o[d] = that sum / l (one division).
+ *
+ * det_oracle_exp(x), defined for x <= 0 (the only arguments step 3 produces):
+ *   x < -104            -> +0.0f
+ *   t = x * LOG2E;  n = rintf(t) (nearest, ties to even);
+ *   f = fmaf(n, -LN2_HI, x);  f = fmaf(n, -LN2_LO, f);                       (|f| <= 0.35)
+ *   p = 1/5040;  p = fmaf(p, f, 1/720);  p = fmaf(p, f, 1/120);  p = fmaf(p, f, 1/24);  p = fmaf(p, f, 1/6);
+ *   p = fmaf(p, f, 1/2);  p = fmaf(p, f, 1);  p = fmaf(p, f, 1);             (Taylor, degree 7)
+ *   result = p * 2^n, as one exact scaling when n >= -126, else (p * 2^(n+64)) * 2^-64 (the second
+ *   multiplication rounds once into the subnormal range).
+ * The constants are the binary32 roundings of log2(e), of the two-term split of ln 2 and of the
+ * reciprocal factorials (bit patterns in the code).  Accurate to within 2 ulp; what matters here is that
+ * the sequence is fixed, so any IEEE-754 implementation reproduces the bits.
+ */
+static float oracle_f32(uint32_t bits)
+{
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+float det_oracle_exp(float x)
+{
+    unsigned mx = oracle_enter_ieee();
+    float r;
+    if (x < -104.0f) {
+        r = 0.0f;
+    } else {
+        const float LOG2E = oracle_f32(0x3FB8AA3Bu);      /* 1.44269502162933349609375        */
+        const float LN2_HI = oracle_f32(0x3F317200u);     /* 0.693145751953125 (low bits zero) */
+        const float LN2_LO = oracle_f32(0x35BFBE8Eu);     /* 1.42860676533018704503775e-06     */
+        const float t = x * LOG2E;
+        const float n = rintf(t);
+        float f = fmaf(n, -LN2_HI, x);
+        f = fmaf(n, -LN2_LO, f);
+        float p = oracle_f32(0x39500D01u);                /* 1/5040 */
+        p = fmaf(p, f, oracle_f32(0x3AB60B61u));          /* 1/720 */
+        p = fmaf(p, f, oracle_f32(0x3C088889u));          /* 1/120 */
+        p = fmaf(p, f, oracle_f32(0x3D2AAAABu));          /* 1/24  */
+        p = fmaf(p, f, oracle_f32(0x3E2AAAABu));          /* 1/6   */
+        p = fmaf(p, f, 0.5f);
+        p = fmaf(p, f, 1.0f);
+        p = fmaf(p, f, 1.0f);
+        const int ni = (int)n;
+        if (ni >= -126) {
+            r = p * oracle_f32((uint32_t)(ni + 127) << 23);
+        } else {
+            const float u = p * oracle_f32((uint32_t)(ni + 64 + 127) << 23);
+            r = u * oracle_f32((uint32_t)(-64 + 127) << 23);
+        }
+    }
+    oracle_leave_ieee(mx);
+    return r;
+}
+
+/* dot product of two length-D vectors in the decode lane order (step 1 above, before the scale) */
+static float oracle_lane_dot(const float *a, const float *b, int64_t D)
+{
+    float acc[32];
+    for (int l = 0; l < 32; ++l) acc[l] = 0.0f;
+    for (int64_t c = 0; c < D; c += 128)
+        for (int l = 0; l < 32; ++l)
+            for (int j = 0; j < 4; ++j) {
+                const int64_t k = c + 4 * (int64_t)l + j;
+                if (k < D) acc[l] = fmaf(a[k], b[k], acc[l]);
+            }
+    for (int w = 32; w > 1; w /= 2)
+        for (int i = 0; i < w / 2; ++i) acc[i] = acc[2 * i] + acc[2 * i + 1];
+    return acc[0];
+}
+
+/* sum of T values in the lane order over j (step 4 above) */
+static float oracle_lane_sum(const float *e, int64_t T)
+{
+    float acc[32];
+    for (int l = 0; l < 32; ++l) acc[l] = 0.0f;
+    for (int64_t c = 0; c < T; c += 128)
+        for (int l = 0; l < 32; ++l)
+            for (int j = 0; j < 4; ++j) {
+                const int64_t k = c + 4 * (int64_t)l + j;
+                if (k < T) acc[l] = acc[l] + e[k];
+            }
+    for (int w = 32; w > 1; w /= 2)
+        for (int i = 0; i < w / 2; ++i) acc[i] = acc[2 * i] + acc[2 * i + 1];
+    return acc[0];
+}
+
+/* the two reductions on their own (exported for the pins) */
+float det_oracle_lane_dot(const float *a, const float *b, int64_t D)
+{
+    unsigned mx = oracle_enter_ieee();
+    const float r = oracle_lane_dot(a, b, D);
+    oracle_leave_ieee(mx);
+    return r;
+}
+
+float det_oracle_lane_sum(const float *e, int64_t T)
+{
+    unsigned mx = oracle_enter_ieee();
+    const float r = oracle_lane_sum(e, T);
+    oracle_leave_ieee(mx);
+    return r;
+}
+
+/* scratch: e [T] floats (caller-provided) */
+static void oracle_attention_one(const float *q, const float *k, const float *v, float scale, int64_t T, int64_t D,
+                                 float *o, float *e)
+{
+    for (int64_t j = 0; j < T; ++j) e[j] = oracle_lane_dot(q, k + j * D, D) * scale;
+    float m = e[0];
+    for (int64_t j = 1; j < T; ++j)
+        if (e[j] > m) m = e[j];
+    for (int64_t j = 0; j < T; ++j) e[j] = det_oracle_exp(e[j] - m);
+    const float l = oracle_lane_sum(e, T);
+    for (int64_t d = 0; d < D; ++d) {
+        float t = 0.0f;
+        for (int64_t j0 = 0; j0 < T; j0 += 256) {
+            const int64_t j1 = j0 + 256 < T ? j0 + 256 : T;
+            float a = 0.0f;
+            for (int64_t j = j0; j < j1; ++j) a = fmaf(e[j], v[j * D + d], a);
+            t = (j0 == 0) ? a : t + a;
+        }
+        o[d] = t / l;
+    }
+}
+
+int det_oracle_attention_decode(const float *q, const float *k, const float *v, float scale, int64_t B, int64_t Hq,
+                                int64_t Hkv, int64_t T, int64_t D, float *o, float *scratch /* [T] per thread: T * threads */)
+{
+    if (!q || !k || !v || !o || !scratch || B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || T < 1 || D < 1) return 1;
+    unsigned mx = oracle_enter_ieee();
+    const int64_t G = Hq / Hkv;
+    int64_t bh;
+#pragma omp parallel for schedule(static)
+    for (bh = 0; bh < B * Hq; ++bh) {
+        unsigned mxt = oracle_enter_ieee();
+        const int64_t b = bh / Hq, h = bh % Hq, hk = h / G;
+#ifdef _OPENMP
+        float *e = scratch + (int64_t)omp_get_thread_num() * T;
+#else
+        float *e = scratch;
+#endif
+        oracle_attention_one(q + (b * Hq + h) * D, k + ((b * Hkv + hk) * T) * D, v + ((b * Hkv + hk) * T) * D, scale, T, D,
+                             o + (b * Hq + h) * D, e);
+        oracle_leave_ieee(mxt);
+    }
+    oracle_leave_ieee(mx);
+    return 0;
+}
+
 int det_oracle_threads(void)
 {
 #ifdef _OPENMP

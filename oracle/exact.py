@@ -185,3 +185,92 @@ def rmsnorm_row(xrow, g, eps: float):
     t = add32(mean, eps)
     r = div32(1.0, sqrt32(t))
     return [mul32(mul32(xv, r), gv) for xv, gv in zip(xrow, g)]
+
+
+# ---- fixed-order decode attention (same definition as the C oracle, on exact rationals) ----------
+def _f32(bits: int) -> float:
+    return struct.unpack("<f", struct.pack("<I", bits))[0]
+
+
+def rint32(t: float) -> float:
+    """Round to the nearest integer, ties to even (what rintf does in the default rounding mode)."""
+    q = Fraction(t)
+    lo = q.numerator // q.denominator
+    rem = q - lo
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and (lo & 1)):
+        lo += 1
+    if lo == 0:
+        return -0.0 if _is_neg(t) else 0.0
+    return float(lo)
+
+
+def exp_det(x: float) -> float:
+    """The attention's exponential for x <= 0: range reduction by ln 2 in two pieces, a degree-7 Taylor
+    polynomial evaluated by Horner's rule with fused multiply-adds, scaling by 2^n (through 2^(n+64) and
+    2^-64 below the normal range); every step one binary32 operation."""
+    if x > 0:
+        raise ValueError("exp_det is defined for x <= 0")
+    if x < -104.0:
+        return 0.0
+    t = mul32(x, _f32(0x3FB8AA3B))
+    n = rint32(t)
+    f = fma32(n, -_f32(0x3F317200), x)
+    f = fma32(n, -_f32(0x35BFBE8E), f)
+    p = _f32(0x39500D01)
+    for c in (_f32(0x3AB60B61), _f32(0x3C088889), _f32(0x3D2AAAAB), _f32(0x3E2AAAAB), 0.5, 1.0, 1.0):
+        p = fma32(p, f, c)
+    ni = int(n)
+    if ni >= -126:
+        return mul32(p, math.ldexp(1.0, ni))
+    return mul32(mul32(p, math.ldexp(1.0, ni + 64)), math.ldexp(1.0, -64))
+
+
+def _lane_tree(acc):
+    w = len(acc)
+    while w > 1:
+        acc = [add32(acc[2 * i], acc[2 * i + 1]) for i in range(w // 2)]
+        w //= 2
+    return acc[0]
+
+
+def lane_dot(a, b) -> float:
+    acc = [0.0] * 32
+    D = len(a)
+    for c in range(0, D, 128):
+        for l in range(32):
+            for j in range(4):
+                k = c + 4 * l + j
+                if k < D:
+                    acc[l] = fma32(a[k], b[k], acc[l])
+    return _lane_tree(acc)
+
+
+def lane_sum(e) -> float:
+    acc = [0.0] * 32
+    T = len(e)
+    for c in range(0, T, 128):
+        for l in range(32):
+            for j in range(4):
+                k = c + 4 * l + j
+                if k < T:
+                    acc[l] = add32(acc[l], e[k])
+    return _lane_tree(acc)
+
+
+def attention_row(q, keys, values, scale: float):
+    """One (batch, head): q [D], keys and values [T][D] (lists of binary32-representable floats)."""
+    T, D = len(keys), len(q)
+    s = [mul32(lane_dot(q, keys[j]), scale) for j in range(T)]
+    m = max(s)
+    e = [exp_det(add32(s[j], -m)) for j in range(T)]
+    l = lane_sum(e)
+    out = []
+    for d in range(D):
+        t = None
+        for j0 in range(0, T, 256):
+            a = 0.0
+            for j in range(j0, min(T, j0 + 256)):
+                a = fma32(e[j], values[j][d], a)
+            t = a if t is None else add32(t, a)
+        out.append(div32(t, l))
+    return out

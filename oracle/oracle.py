@@ -105,6 +105,14 @@ def lib() -> ctypes.CDLL:
         L.det_oracle_sum_squares.restype = ctypes.c_float
         L.det_oracle_rmsnorm.argtypes = [p, p, ctypes.c_float, i64, i64, p]
         L.det_oracle_rmsnorm.restype = i32
+        L.det_oracle_exp.argtypes = [ctypes.c_float]
+        L.det_oracle_exp.restype = ctypes.c_float
+        L.det_oracle_attention_decode.argtypes = [p, p, p, ctypes.c_float, i64, i64, i64, i64, i64, p, p]
+        L.det_oracle_attention_decode.restype = i32
+        L.det_oracle_lane_dot.argtypes = [p, p, i64]
+        L.det_oracle_lane_dot.restype = ctypes.c_float
+        L.det_oracle_lane_sum.argtypes = [p, i64]
+        L.det_oracle_lane_sum.restype = ctypes.c_float
         _lib = L
     return _lib
 
@@ -205,6 +213,43 @@ def rmsnorm(x, g, eps: float):
     if rc != 0:
         raise ValueError("det_oracle_rmsnorm rejected its arguments")
     return y
+
+
+def exp_det(x: float) -> float:
+    """The fixed-sequence exponential of the attention (defined for x <= 0)."""
+    return float(lib().det_oracle_exp(float(np.float32(x))))
+
+
+def lane_dot(a, b) -> float:
+    """Dot product in the decode lane order (the attention's q . k_j before the scale)."""
+    a = np.ascontiguousarray(a, dtype=np.float32).reshape(-1)
+    b = np.ascontiguousarray(b, dtype=np.float32).reshape(-1)
+    assert a.size == b.size
+    return float(lib().det_oracle_lane_dot(a.ctypes.data, b.ctypes.data, a.size))
+
+
+def lane_sum(e) -> float:
+    """Sum in the lane order over the keys (the attention's softmax denominator)."""
+    e = np.ascontiguousarray(e, dtype=np.float32).reshape(-1)
+    return float(lib().det_oracle_lane_sum(e.ctypes.data, e.size))
+
+
+def attention_decode(q, k, v, scale: float):
+    """Fixed-order decode attention: q [B,Hq,D], k and v [B,Hkv,T,D] float32 -> o [B,Hq,D]; one query row
+    per (batch, head) against T cached keys and values, grouped-query heads when Hq > Hkv."""
+    q = np.ascontiguousarray(q, dtype=np.float32)
+    k = np.ascontiguousarray(k, dtype=np.float32)
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    B, Hq, D = q.shape
+    Bk, Hkv, T, Dk = k.shape
+    assert (Bk, Dk) == (B, D) and v.shape == k.shape and Hq % Hkv == 0
+    o = np.empty((B, Hq, D), dtype=np.float32)
+    scratch = np.empty(T * max(1, int(lib().det_oracle_threads())), dtype=np.float32)
+    rc = lib().det_oracle_attention_decode(q.ctypes.data, k.ctypes.data, v.ctypes.data, float(np.float32(scale)),
+                                           B, Hq, Hkv, T, D, o.ctypes.data, scratch.ctypes.data)
+    if rc != 0:
+        raise ValueError("det_oracle_attention_decode rejected its arguments")
+    return o
 
 
 def up(h: int) -> float:
