@@ -49,7 +49,7 @@ typedef enum {
     DET_OK = 0,
     DET_ERR_INVALID_ARG = 1,        /* NULL pointer, non-positive size, buffer too small          */
     DET_ERR_UNSUPPORTED_SHAPE = 2,  /* a dimension exceeds what the kernels index (see below)     */
-    DET_ERR_ALIGNMENT = 3,          /* reserved: misaligned buffers take the generic kernel       */
+    DET_ERR_ALIGNMENT = 3,          /* a buffer misses the alignment an entry point without a generic path needs */
     DET_ERR_ALLOC = 4,              /* device or host allocation failed                           */
     DET_ERR_CUDA = 5,               /* a CUDA call failed; det_last_error() has the message       */
     DET_ERR_DEVICE_TIMEOUT = 6,     /* a kernel gave up a bounded wait (see det_linear_plan_check)*/
@@ -226,6 +226,32 @@ DET_API det_status_t det_argmax_rows(const float* y, int64_t M, int64_t N, int32
  */
 DET_API det_status_t det_rmsnorm(const float* x, const float* g, float eps, int64_t M, int64_t H, float* y,
                                  void* stream);
+
+/*
+ * Fixed-order decode attention: o[b,h,:] = softmax_j(q[b,h,:] . k[b,h',j,:] * scale) . v[b,h',:,:] for one
+ * query row per (batch, head) against T cached keys and values, h' = h / (Hq / Hkv) (grouped-query heads).
+ * An extension, not one of the paper's kernels: the paper keeps vendor attention and names fixed-order
+ * attention as the outstanding source of residual divergence between GPU architectures.  Every step is
+ * one IEEE binary32 operation in an order fixed by (T, D) alone:
+ *   s_j = dot(q, k_j) * scale, the dot product in the decode lane order of this header over D (chunks of
+ *         128 ascending, lane l owns 4 consecutive elements, one fmaf per element from +0.0f, elements
+ *         beyond D skipped, adjacent-first 32-lane tree), then one multiply;
+ *   m   = max_j s_j;   e_j = exp_det(s_j - m), exp_det a fixed sequence of binary32 operations (range
+ *         reduction by ln 2 in two pieces, degree-7 Taylor polynomial by Horner's rule with fmaf, exact
+ *         scaling by 2^n; within 2 ulp of the real exponential; +0 below -104);
+ *   l   = sum_j e_j in the lane order over j (chunks of 128 keys, lane l owns 4 consecutive keys, one add
+ *         per key from +0.0f, adjacent-first tree);
+ *   o_d = (sum over 256-key segments, ascending, of the chain a = fmaf(e_j, v_j[d], a) from +0.0f) / l.
+ * The bits do not depend on B, the grid, the stream or the SM count.
+ *   q : device FP32 [B, Hq, D];  k, v : device FP32 [B, Hkv, T, D];  o : device FP32 [B, Hq, D]; all
+ *   row-major, contiguous and 16-byte aligned (DET_ERR_ALIGNMENT otherwise).
+ *   Hq / Hkv in {1, 2, 4, 8}; D a multiple of 4, at most 256; the scores and segment sums of a (batch,
+ *   KV head) live in shared memory, which limits T (about 9000 keys at Hq / Hkv = 4, D = 128):
+ *   DET_ERR_UNSUPPORTED_SHAPE with a message beyond that.
+ * Enqueued on `stream`, no synchronisation, no allocation.
+ */
+DET_API det_status_t det_attention_decode(const float* q, const float* k, const float* v, float scale, int64_t B,
+                                          int64_t Hq, int64_t Hkv, int64_t T, int64_t D, float* o, void* stream);
 
 /*
  * The same computation for callers that cannot allocate (the paper has no counterpart for this

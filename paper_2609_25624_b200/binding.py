@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.det_argmax_rows.restype = i32
         L.det_rmsnorm.argtypes = [p, p, ctypes.c_float, i64, i64, p, p]
         L.det_rmsnorm.restype = i32
+        L.det_attention_decode.argtypes = [p, p, p, ctypes.c_float, i64, i64, i64, i64, i64, p, p]
+        L.det_attention_decode.restype = i32
         L.det_last_error.restype = ctypes.c_char_p
         L.det_order_version.restype = i32
         L.det_last_status.restype = i32
@@ -319,6 +321,18 @@ def det_rmsnorm(x, g, eps: float, y, stream=None) -> None:
     _expect(g, torch.float32, (H,), "g")
     _expect(y, torch.float32, (M, H), "y")
     _check(lib().det_rmsnorm(x.data_ptr(), g.data_ptr(), float(eps), M, H, y.data_ptr(), _stream_ptr(stream)))
+
+
+def det_attention_decode(q, k, v, scale: float, o, stream=None) -> None:
+    """Fixed-order decode attention: q [B,Hq,D], k and v [B,Hkv,T,D], o [B,Hq,D], float32 CUDA tensors."""
+    B_, Hq, D = q.shape
+    Bk, Hkv, T, Dk = k.shape
+    _expect(q, torch.float32, (B_, Hq, D), "q")
+    _expect(k, torch.float32, (B_, Hkv, T, D), "k")
+    _expect(v, torch.float32, (B_, Hkv, T, D), "v")
+    _expect(o, torch.float32, (B_, Hq, D), "o")
+    _check(lib().det_attention_decode(q.data_ptr(), k.data_ptr(), v.data_ptr(), float(scale), B_, Hq, Hkv, T, D,
+                                      o.data_ptr(), _stream_ptr(stream)))
 
 
 def det_argmax_rows(y, idx, stream=None) -> None:

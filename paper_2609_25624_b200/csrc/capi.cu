@@ -290,6 +290,40 @@ det_status_t det_rmsnorm(const float* x, const float* g, float eps, int64_t M, i
     return DET_OK;
 }
 
+det_status_t det_attention_decode(const float* q, const float* k, const float* v, float scale, int64_t B, int64_t Hq, int64_t Hkv,
+                                  int64_t T, int64_t D, float* o, void* stream)
+{
+    if (!q || !k || !v || !o) { set_error("attention: q, k, v and o must not be NULL"); return DET_ERR_INVALID_ARG; }
+    if (B < 1 || Hq < 1 || Hkv < 1 || T < 1 || D < 1 || Hq % Hkv != 0 || B * Hkv >= (1ll << 31) || T >= (1ll << 24)) {
+        set_error("attention: need B, Hq, Hkv, T, D >= 1, Hq a multiple of Hkv, B * Hkv < 2^31, T < 2^24");
+        return DET_ERR_INVALID_ARG;
+    }
+    const int64_t G = Hq / Hkv;
+    if ((G != 1 && G != 2 && G != 4 && G != 8) || D % 4 != 0 || D > 256) {
+        set_error("attention: this kernel serves 1, 2, 4 or 8 query heads per KV head and head dimensions that are multiples of 4 up to 256 "
+                  "(got Hq / Hkv = %lld, D = %lld)", (long long)G, (long long)D);
+        return DET_ERR_UNSUPPORTED_SHAPE;
+    }
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) {
+        set_error("attention: q, k, v and o must be 16-byte aligned");
+        return DET_ERR_ALIGNMENT;
+    }
+    const size_t smem = attention_smem_bytes((int)G, (int)T, (int)D);
+    if (smem > 227u * 1024u) {
+        set_error("attention: T = %lld keys with %lld query heads per KV head need %zu bytes of shared memory for the scores and the "
+                  "segment sums; a thread block has %u", (long long)T, (long long)G, smem, 227u * 1024u);
+        return DET_ERR_UNSUPPORTED_SHAPE;
+    }
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail("attention: device query", e);
+    if (major != 10) { set_error("attention: device %d is sm_%dx; this library is built for sm_100a only", dev, major); return DET_ERR_ARCH; }
+    e = launch_attention_decode(q, k, v, scale, (int)B, (int)Hq, (int)Hkv, (int)T, (int)D, o, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail("attention: launch", e);
+    return DET_OK;
+}
+
 det_status_t det_linear_plan_tune(det_linear_plan_t* plan, const float* x, const void* W, const float* b, float* y,
                                   void* stream, int32_t* variant_out, float* best_us_out)
 {

@@ -58,6 +58,10 @@ cudaError_t launch_prefill(const LaunchArgs& a);
 int prefill_rows_per_thread(int64_t M);
 // Fixed-order RMSNorm of M rows of H elements (rmsnorm.cu).
 cudaError_t launch_rmsnorm(const float* x, const float* g, float eps, int64_t M, int64_t H, float* y, cudaStream_t stream);
+// Fixed-order decode attention (attention.cu); attention_smem_bytes = dynamic shared memory it needs.
+size_t attention_smem_bytes(int G, int T, int D);
+cudaError_t launch_attention_decode(const float* q, const float* k, const float* v, float scale, int B, int Hq, int Hkv, int T,
+                                    int D, float* o, cudaStream_t stream);
 // Read `bytes` at buf through L2 (evicts what was there without leaving dirty lines); sink: 4 bytes of device memory.
 cudaError_t launch_l2_evict(const void* buf, size_t bytes, unsigned* sink, int sm_count, cudaStream_t stream);
 cudaError_t launch_argmax(const float* y, int64_t M, int64_t N, int32_t* idx, cudaStream_t stream);
