@@ -350,6 +350,7 @@ def run_own(args, world, rank, local):
         tables["column_shards"] = shard_table(B, dev, st, hbm_peak)
         tables["r3_ablation"] = ablation_table(B, dev, st)
         tables["rmsnorm"] = rmsnorm_table(B, dev, st, hbm_peak)
+        tables["attention"] = attention_table(B, dev, st, hbm_peak)
     for w in work:                       # free the sweep's 2.2 GB (before the 15 GB stack)
         w["plan"].close()
     work.clear()
@@ -619,6 +620,31 @@ def rmsnorm_table(B, dev, st, hbm_peak):
     return rows
 
 
+def attention_table(B, dev, st, hbm_peak):
+    """Fixed-order decode attention with the Llama-3-8B head geometry (32 query heads, 8 KV heads, D = 128,
+    FP32 cache): algorithmic bytes = K and V once (8 B Hkv T D) + q + o.  One thread block per (batch, KV head)."""
+    import math
+    Hq, Hkv, D = 32, 8, 128
+    rows = []
+    for (Bt, T) in ((1, 4096), (8, 4096), (32, 2048), (32, 8192)):
+        g = torch.Generator().manual_seed(Bt * 131 + T)
+        q = torch.randn(Bt, Hq, D, generator=g).to(dev)
+        k = torch.randn(Bt, Hkv, T, D, generator=g).to(dev)
+        v = torch.randn(Bt, Hkv, T, D, generator=g).to(dev)
+        o = torch.empty_like(q)
+        scale = 1.0 / math.sqrt(D)
+        with torch.cuda.stream(st):
+            B.det_attention_decode(q, k, v, scale, o)
+            torch.cuda.synchronize()
+        reps = 4
+        ms = time_graph(lambda: [B.det_attention_decode(q, k, v, scale, o) for _ in range(reps)], 3, st) / reps
+        nbytes = 8 * Bt * Hkv * T * D + 8 * Bt * Hq * D
+        rows.append({"B": Bt, "Hq": Hq, "Hkv": Hkv, "T": T, "D": D, "blocks": Bt * Hkv, "us": ms * 1e3,
+                     "gbs": nbytes / ms / 1e6, "pct_hbm": 100 * nbytes / ms / 1e6 / hbm_peak,
+                     "l2_resident": nbytes < (100 << 20)})
+    return rows
+
+
 def lm_head_table(B, dev, st, hbm_peak, fp32_peak):
     name, K, N = inputs.LLAMA3_8B_LM_HEAD
     rows = []
@@ -733,8 +759,28 @@ def cpu_baseline(passes=8):
 def run_case(args):
     """One shape, few launches: the workload used for ncu captures of a single kernel."""
     from paper_2609_25624_b200 import binding as B
-    dims = [int(v) for v in args.case.split(",")]
     torch.cuda.set_device(0)
+    if args.case.startswith("attn:"):         # attn:B,T -- a few det_attention_decode launches (Llama-3-8B head geometry)
+        import math
+        Bt, T = (int(v) for v in args.case[5:].split(","))
+        g = torch.Generator().manual_seed(Bt * 131 + T)
+        q = torch.randn(Bt, 32, 128, generator=g).cuda()
+        k = torch.randn(Bt, 8, T, 128, generator=g).cuda()
+        v = torch.randn(Bt, 8, T, 128, generator=g).cuda()
+        o = torch.empty_like(q)
+        for _ in range(3):
+            B.det_attention_decode(q, k, v, 1.0 / math.sqrt(128), o)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            B.det_attention_decode(q, k, v, 1.0 / math.sqrt(128), o)
+        e1.record()
+        torch.cuda.synchronize()
+        print(json.dumps({"case": ["attention", Bt, 32, 8, T, 128], "launches": args.steps, "warmup_launches": 3,
+                          "us_per_launch_eager": e0.elapsed_time(e1) * 1e3 / args.steps}), flush=True)
+        return
+    dims = [int(v) for v in args.case.split(",")]
     if len(dims) == 2:                       # M,H: the fixed-order RMSNorm kernel
         M, H = dims
         x = torch.randn(M, H, generator=torch.Generator().manual_seed(M)).cuda()
@@ -784,8 +830,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the per-case, prefill and LM-head tables")
     ap.add_argument("--tables", default=None, metavar="PATH", help="also write the long per-case tables (JSON) to this file")
     ap.add_argument("--ref-cols", type=int, default=ORACLE_SAMPLE_ROWS, help="weight rows per case in the reference arm's sample")
-    ap.add_argument("--case", default=None, metavar="M,N,K | M,H",
-                    help="M,H: a few det_rmsnorm launches.  M,N,K: run only this shape: --steps eager det_linear_run calls over rotating weight copies "
+    ap.add_argument("--case", default=None, metavar="M,N,K | M,H | attn:B,T",
+                    help="attn:B,T: a few det_attention_decode launches.  M,H: a few det_rmsnorm launches.  M,N,K: run only this shape: --steps eager det_linear_run calls over rotating weight copies "
                          "(a small, profiler-friendly workload; prints its own one-line JSON)")
     args = ap.parse_args()
     if args.case:

@@ -41,6 +41,7 @@ static const DecodeEntry kEntries2[] = {
     ROW(4, 1, 14, 3, 2, 256),
     ROW(2, 2, 14, 2, 2, 256),
     ROW(2, 2, 14, 2, 2, 512),
+    ROW(2, 2, 14, 1, 2, 256),
     ROW(4, 1, 14, 2, 1, 256),
     ROW(4, 1, 14, 4, 1, 256),
 };

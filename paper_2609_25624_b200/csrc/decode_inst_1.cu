@@ -19,6 +19,7 @@ using namespace decode_detail;
 static const DecodeEntry kEntries3[] = {
     ROW(4, 2, 14, 2, 2, 256),
     ROW(4, 2, 14, 2, 2, 512),
+    ROW(4, 2, 14, 1, 2, 256),
     ROW(8, 1, 14, 3, 2, 256),
     ROW(8, 1, 14, 4, 2, 256),
     ROW(8, 1, 14, 2, 2, 256),

@@ -18,6 +18,7 @@ using namespace decode_detail;
 
 static const DecodeEntry kEntries4[] = {
     ROW(8, 2, 14, 2, 2, 256),
+    ROW(8, 2, 14, 1, 2, 256),
     ROW(8, 2, 14, 2, 1, 256),
     ROW(8, 2, 14, 4, 1, 256),
     ROW(8, 2, 14, 4, 1, 512),

@@ -474,10 +474,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                 };
                 if (k0 + KC <= k_hi) {
                     // whole stage inside the segment: no per-lane test
+                    {
 #pragma unroll(MT * RT >= 64 ? 1 : 2)
-                    for (int cc = 0; cc < KC / 128 - 1; ++cc) chunk(cc);
-                    ready = mbar_test_wait(fullg + 8 * st, phase);          // look ahead: the stage after this one
-                    chunk(KC / 128 - 1);
+                        for (int cc = 0; cc < KC / 128 - 1; ++cc) chunk(cc);
+                        ready = mbar_test_wait(fullg + 8 * st, phase);          // look ahead: the stage after this one
+                        chunk(KC / 128 - 1);
+                    }
                 } else {
                     ready = false;
                     // Last stage of a ragged K: elements beyond the end are skipped, not zero-filled
