@@ -161,12 +161,18 @@ template <int MT, int WM, int RT, int WR, int SK, int KC, int STAGES, int WF>
 struct Cfg {
     static constexpr int kGroupWarps = WM * WR;               // consumer warps that share one ring
     static constexpr int kConsumerWarps = SK * kGroupWarps;
-    // Producers: one warp per segment group.  Where the consumers hold 8-row register tiles in whole
-    // warpgroups, the producers fill a warpgroup of their own and the kernel moves registers from them to
-    // the consumers with setmaxnreg: the register file is split over the four schedulers, so nine or ten
-    // warps per SM would cap every thread at 168 registers, less than an 8 x 14 tile needs.
+    // Producers: two warps per segment group, one requesting the weight tiles and one the activation tiles
+    // (a bulk-tensor request costs its issuing thread some 200 cycles, and the activations can only be
+    // requested once the previous kernel in the stream has finished).  Where the consumers hold 8-row
+    // register tiles in whole warpgroups, the producers fill a warpgroup of their own and the kernel moves
+    // registers from them to the consumers with setmaxnreg: the register file is split over the four
+    // schedulers, so nine or ten warps per SM would cap every thread at 168 registers, less than an 8 x 14
+    // tile needs.
     static constexpr bool kMoveRegs = (MT == 8 && (kConsumerWarps == 4 || kConsumerWarps == 8));
-    static constexpr int kPG = kMoveRegs ? 4 : SK;
+    // (8-row tiles in six consumer warps keep a single producer warp per group, which then requests both:
+    // a tenth warp would bring the 168-register cap back.)
+    static constexpr bool kSplitProducers = kMoveRegs || MT < 8;
+    static constexpr int kPG = kMoveRegs ? 4 : (kSplitProducers ? 2 * SK : SK);
     static constexpr int kThreads = (kConsumerWarps + kPG) * 32;   // the producer group comes last
     static constexpr int kMB = MT * WM;                       // batch rows per x box
     static constexpr int kRB = RT * WR;                       // weight rows per W box (= per work unit)
@@ -201,7 +207,7 @@ struct Cfg {
     static_assert(!kMoveRegs || kConsumerRegs * kConsumerWarps * 32 + kProducerRegs * kPG * 32 <= kThreads * kLaunchRegs,
                   "register move must fit in the block's own allocation");
     static_assert(!kMoveRegs || kConsumerRegs >= kLaunchRegs, "consumers only ever grow");
-    static_assert(SK <= 4, "one producer warp per segment group");
+    static_assert((kSplitProducers ? 2 : 1) * SK <= kPG, "one or two producer warps per segment group");
     // shared memory of a launch whose order has S segments (the S partial tiles when SK > 1)
     static constexpr int smem_bytes(int S) { return kFixedSmem + (SK > 1 ? S * kTile * 4 : 0); }
     static_assert(RT % 2 == 0, "weight rows are processed in pairs (one FP32x2 accumulator per pair)");
@@ -260,14 +266,16 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         const int pg = warp - C::kConsumerWarps;
         if (pg < SK && lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
             for (int i = 0; i < STAGES; ++i) {
                 mbar_init(full0 + 8 * (pg * STAGES + i), 1);
                 mbar_init(empty0 + 8 * (pg * STAGES + i), C::kGroupWarps);
             }
             if (pg == 0) sts_volatile_i32(abort_flag, 0);
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            // make the initialised barriers visible to the bulk-copy engine
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (!C::kSplitProducers) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        } else if (C::kSplitProducers && pg < 2 * SK && lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
         }
         __syncwarp();
         asm volatile("bar.arrive 2, %0;" ::"r"(C::kThreads) : "memory");
@@ -287,10 +295,14 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     };
 
     if (warp >= C::kConsumerWarps) {
-        // ---------------- producers: lane 0 of producer warp g issues the bulk-tensor copies of group g ----------------
+        // ---------------- producers: lane 0 of producer warp g requests the weight tiles of group g, lane 0 of
+        // producer warp SK + g its activation tiles ----------------
         if (C::kMoveRegs) reg_dec<C::kProducerRegs>();
-        const int g = warp - C::kConsumerWarps;
-        if (g >= SK || lane != 0) return;
+        const int pw = warp - C::kConsumerWarps;
+        if (pw >= (C::kSplitProducers ? 2 : 1) * SK || lane != 0) return;
+        const bool do_x = !C::kSplitProducers || pw >= SK;          // requests activation tiles
+        const bool do_w = !C::kSplitProducers || pw < SK;           // requests weight tiles
+        const int g = pw >= SK ? pw - SK : pw;
         unsigned long long pol_w, pol_x;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_w));
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_x));
@@ -324,51 +336,54 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             seg_range(c.r * SK + g, c.k0, c.k_hi);
             return true;
         };
-        auto issue_w = [&](int st, const Cursor& c) {
+        // The weight producer announces the stage's bytes (weights and activations) on its full barrier;
+        // the activation producer only adds its copy (the byte count of a barrier may run ahead of the
+        // announcement: the phase cannot complete before the announcing arrival).
+        auto issue = [&](int st, const Cursor& c, bool w, bool x) {
             const uint32_t fb = fullg + 8 * st;
-            mbar_arrive_expect_tx(fb, C::kStageBytes);
+            if (w) mbar_arrive_expect_tx(fb, C::kStageBytes);
 #pragma unroll
-            for (int sub = 0; sub < C::kSubs; ++sub)
-                tma_load_2d(ringg + (uint32_t)(st * C::kStageBytes + sub * C::kSubBytes) + C::kXBytes, &map_w, c.k0 + sub * C::kKB,
-                            c.tile * C::kRB, fb, pol_w);
-        };
-        auto issue_x = [&](int st, const Cursor& c) {
-#pragma unroll
-            for (int sub = 0; sub < C::kSubs; ++sub)
-                tma_load_2d(ringg + (uint32_t)(st * C::kStageBytes + sub * C::kSubBytes), &map_x, c.k0 + sub * C::kKB, c.mb * C::kMB,
-                            fullg + 8 * st, pol_x);
+            for (int sub = 0; sub < C::kSubs; ++sub) {
+                const uint32_t dst = ringg + (uint32_t)(st * C::kStageBytes + sub * C::kSubBytes);
+                if (w) tma_load_2d(dst + C::kXBytes, &map_w, c.k0 + sub * C::kKB, c.tile * C::kRB, fb, pol_w);
+                if (x) tma_load_2d(dst, &map_x, c.k0 + sub * C::kKB, c.mb * C::kMB, fb, pol_x);
+            }
         };
 
-        // Weights never depend on the previous kernel in the stream, activations may: the first ring
-        // of weight boxes is requested before waiting for that kernel to finish.
         Cursor c;
         bool live = start(c);
+        // Weights never depend on the previous kernel in the stream, activations may: weight requests start at
+        // once, activation requests wait for that kernel to finish.  A thread that requests both sends the
+        // first ring of weight requests ahead of the wait.
         int pre = 0;
-        while (live && pre < STAGES) {
-            issue_w(pre, c);
-            ++pre;
-            live = advance(c);
+        if (do_w && do_x) {
+            const Cursor c0 = c;
+            const bool live0 = live;
+            while (live && pre < STAGES) {
+                issue(pre, c, true, false);
+                ++pre;
+                live = advance(c);
+            }
+            c = c0;
+            live = live0;
         }
-        pdl_wait();
-
-        live = start(c);
+        if (do_x) pdl_wait();
         int st = 0;
         unsigned phase = 0, n_issued = 0;
         bool ok = true;
         while (live) {
-            if ((int)n_issued >= pre) {
+            if (n_issued >= (unsigned)STAGES) {
                 // the slot's previous use must have been released by every consumer warp of the group
                 if (!mbar_wait(emptyg + 8 * st, phase ^ 1, abort_flag, status, wait_limit_ns, 1)) { ok = false; break; }
-                issue_w(st, c);
             }
             const bool withhold = (test_flags & kTestWithholdFirstX) && blockIdx.x == 0 && g == 0 && n_issued == 0;
-            if (!withhold) issue_x(st, c);
+            issue(st, c, do_w && (int)n_issued >= pre, do_x && !withhold);
             ++n_issued;
             if (++st == STAGES) { st = 0; phase ^= 1; }
             live = advance(c);
         }
         if (!ok) {
-            // aborting: wait (bounded) for the copies this thread still has in flight
+            // aborting: wait (bounded) for the copies still in flight in the group's ring
             const unsigned first = n_issued > (unsigned)STAGES ? n_issued - STAGES : 0u;
             for (unsigned j = first; j < n_issued; ++j) {
                 const unsigned long long t0 = global_timer_ns();
@@ -579,6 +594,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
 
         if constexpr (SK > 1) {
             // ---- fold the S segment sums of every output in ascending order, bias last, store ----
+            // (the bias of the thread's first output is requested before the barrier: its latency hides there)
+            float b_first = 0.0f;
+            {
+                const int n = tile * C::kRB + (int)threadIdx.x % C::kRB;
+                if (bias != nullptr && (int)threadIdx.x < C::kTile && n < N) b_first = __ldg(bias + n);
+            }
             consumer_barrier(C::kConsumerWarps * 32);
             const bool aborting = lds_volatile_i32(abort_flag) != 0;
             if (!waited) { pdl_wait(); waited = true; }
@@ -589,7 +610,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                     if (m < M && n < N) {
                         float t = part[o];
                         for (int s2 = 1; s2 < S; ++s2) t = __fadd_rn(t, part[s2 * C::kTile + o]);
-                        if (bias) t = __fadd_rn(t, __ldg(bias + n));
+                        if (bias) t = __fadd_rn(t, o == (int)threadIdx.x ? b_first : __ldg(bias + n));
                         y[(long long)m * ldy + n] = t;
                     }
                 }

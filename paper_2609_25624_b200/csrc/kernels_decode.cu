@@ -42,15 +42,15 @@ double tiling_cost(const DecodeEntry& e, int64_t M, int64_t N, int64_t K, int S,
     const int64_t per_sm = (units + sm_count - 1) / sm_count;
     const double resident = (double)(per_sm < occ ? per_sm : occ);
     const double warps = resident * c.wm * c.wr * c.sk;
-    double eff = c.mt >= 8 ? 0.735 : c.mt == 4 ? 0.70 : c.mt == 2 ? 0.345 : 0.2;
+    double eff = c.mt >= 8 ? 0.707 : c.mt == 4 ? 0.70 : c.mt == 2 ? 0.345 : 0.2;
     if (c.kc >= 512 && c.mt >= 8) eff *= 1.2;          // half as many stage boundaries; smaller tiles prefer a deeper ring
     if (c.kc <= 128) eff *= 0.9;
-    const double latency = warps >= 8.0 ? 1.0 : sqrt(8.0 / warps);
+    const double latency = warps >= 8.0 ? 1.0 : 8.0 / warps;
     const double fma = (double)rb * (double)mb * (double)K / 128.0 / eff * resident;
     // weights from HBM at 22.5 bytes per clock and SM; the unit's activations come again from L2 for every unit
     const double hbm = ((double)rb * (double)K * 2.0 / 22.5 + 0.06 * (double)mb * (double)K * 4.0 / 64.0) * resident;
     const double body = (fma > hbm ? fma : hbm) * latency;
-    const double overhead = (double)S * 1100.0 * ((double)(mb * rb) / 896.0) + (c.sk > 1 ? 1500.0 : 0.0);
+    const double overhead = (double)S * 1020.0 * ((double)(mb * rb) / 896.0) + (c.sk > 1 ? 1500.0 : 0.0);
     return (double)rounds * (body + overhead);
 }
 
