@@ -16,7 +16,7 @@ OBJ_DIR = os.path.join(HERE, "csrc", "obj")
 
 # (source, extra defines): the decode tilings are compiled once per weight format
 SOURCES = [("plan.cpp", ()), ("capi.cu", ()), ("kernels_generic.cu", ()), ("kernels_decode.cu", ()),
-           ("kernels_prefill.cu", ()), ("bench_kernels.cu", ()), ("noalloc.cu", ()), ("ablation.cu", ()), ("rmsnorm.cu", ()), ("attention.cu", ())]
+           ("kernels_prefill.cu", ()), ("prefill_tma.cu", ()), ("bench_kernels.cu", ()), ("noalloc.cu", ()), ("ablation.cu", ()), ("rmsnorm.cu", ()), ("attention.cu", ())]
 SOURCES += [(f"decode_inst_{i}.cu", (f"-DDET_WF={wf}",)) for wf in (0, 1, 2) for i in range(4)]
 
 NVCC_FLAGS = [

@@ -43,7 +43,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 // 2-D row-major tensor [rows, cols] of `elem_bytes`-wide elements, box [box_rows, box_cols].
 static bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t rows,
-                      uint64_t cols, uint32_t box_rows, uint32_t box_cols, CUtensorMapL2promotion promo)
+                      uint64_t cols, uint32_t box_rows, uint32_t box_cols, CUtensorMapL2promotion promo,
+                      CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE)
 {
     static EncodeTiledFn encode = driver_fn<EncodeTiledFn>("cuTensorMapEncodeTiled");
     if (!encode) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return false; }
@@ -52,7 +53,7 @@ static bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, 
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = encode(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_NONE, promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                        swizzle, promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r); return false; }
     return true;
 }
@@ -123,7 +124,30 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const vo
         }
         e = launch_decode(a, cfg, &plan->map_w, &plan->map_x);
     } else if (kernel == kKernelPrefill) {
-        e = launch_prefill(a);
+        // 16-bit weights: the TMA-fed kernel (variant 5 .. 8 forces its rows per thread); FP32 weights, or
+        // variant 15 .. 18, the register-staged kernel
+        const int v = plan->variant;
+        if (!plan->x_t || (v >= 15 && v <= 18)) {
+            e = launch_prefill(a);
+        } else {
+            const int tr = (v >= 5 && v <= 8) ? v : prefill_rows_per_thread(p.M);
+            const int cfg_id = 4096 + tr + 1024 * p.weight_format;
+            const int64_t ldt = (p.M + 3) / 4 * 4;
+            e = launch_transpose_x(x, plan->x_t, p.M, p.K, ldt, stream);
+            if (e != cudaSuccess) return cuda_fail("kernel launch", e);
+            if (plan->map_w_ptr != W || plan->map_cfg_id != cfg_id) {
+                const CUtensorMapDataType wdt = p.weight_format == DET_WEIGHT_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                                                   : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+                if (!encode_2d(&plan->map_w, wdt, 2, W, (uint64_t)plan->n_count, (uint64_t)p.K, 128u, 32u,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+                    return DET_ERR_CUDA;
+                if (!encode_2d(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, plan->x_t, (uint64_t)p.K, (uint64_t)ldt, 32u,
+                               (uint32_t)(16 * tr), CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+                    return DET_ERR_CUDA;
+                plan->map_w_ptr = W; plan->map_x_ptr = plan->x_t; plan->map_cfg_id = cfg_id;
+            }
+            e = launch_prefill_tma(a, tr, &plan->map_w, &plan->map_x);
+        }
     } else {
         e = launch_generic(a, p.bucket);
     }
@@ -201,6 +225,12 @@ det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K, int64_
         cudaGetLastError();
         det_linear_plan_destroy(plan);              // frees whatever was allocated before the failure
         return nullptr;
+    }
+    // Activation workspace of the TMA-fed prefill kernel (16-bit weights): x transposed, 4 K roundup(M, 4) bytes.
+    // Without it the plan still works: it uses the register-staged kernel, which computes the same bits.
+    if (prm.kernel == kKernelPrefill && wfmt != DET_WEIGHT_FP32) {
+        e = device_alloc(reinterpret_cast<void**>(&plan->x_t), 4ull * (uint64_t)((M + 3) / 4 * 4) * (uint64_t)K);
+        if (e != cudaSuccess) { plan->x_t = nullptr; cudaGetLastError(); }
     }
     return plan;
 }
@@ -415,10 +445,12 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
                      "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"sk\": %d, \"kc\": %d, \"stages\": %d, \"blocks_per_sm\": %d}",
                      c.mt, c.wm, c.rt, c.wr, c.sk, c.kc, c.stages, decode_config_occupancy(p.weight_format, c, p.S));
     }
-    char ptile[64] = "null";
+    char ptile[96] = "null";
     if (p.kernel == kKernelPrefill) {
-        const int tr = (plan->variant >= 5 && plan->variant <= 8) ? plan->variant : prefill_rows_per_thread(p.M);
-        snprintf(ptile, sizeof ptile, "{\"bm\": %d, \"bn\": 128, \"bk\": 32}", 16 * tr);
+        const int v = plan->variant;
+        const bool staged = !plan->x_t || (v >= 15 && v <= 18);
+        const int tr = (v >= 5 && v <= 8) ? v : (v >= 15 && v <= 18) ? v - 10 : prefill_rows_per_thread(p.M);
+        snprintf(ptile, sizeof ptile, "{\"bm\": %d, \"bn\": 128, \"bk\": 32, \"feed\": \"%s\"}", 16 * tr, staged ? "registers" : "tma");
     }
     int w = snprintf(buf, n,
                      "{\"M\": %lld, \"N\": %lld, \"K\": %lld, \"bucket\": \"%s\", \"V\": %d, \"L\": %d, \"P\": %d, "
@@ -437,6 +469,7 @@ void det_linear_plan_destroy(det_linear_plan_t* plan)
 {
     if (!plan) return;
     if (plan->partials) cudaFree(plan->partials);
+    if (plan->x_t) cudaFree(plan->x_t);
     if (plan->status) cudaFree(plan->status);
     if (plan->x_stage) cudaFree(plan->x_stage);
     if (plan->y_stage) cudaFree(plan->y_stage);
@@ -489,8 +522,9 @@ det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
             set_error("set_variant: the decode kernel has fewer than %d tilings for this batch size", variant);
             return DET_ERR_INVALID_ARG;
         }
-    } else if (variant != 0 && (variant < 5 || variant > 8)) {
-        set_error("set_variant: the prefill kernel takes 0 (automatic) or 5 .. 8 rows per thread");
+    } else if (variant != 0 && (variant < 5 || variant > 8) && (variant < 15 || variant > 18)) {
+        set_error("set_variant: the prefill bucket takes 0 (automatic), 5 .. 8 (rows per thread) or 15 .. 18 (the same with "
+                  "the register-staged kernel)");
         return DET_ERR_INVALID_ARG;
     }
     plan->variant = variant;

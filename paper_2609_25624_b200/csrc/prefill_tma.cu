@@ -1,0 +1,331 @@
+// Prefill kernel for 16-bit weights (bucket M > 64): register-tiled FP32 GEMM on the CUDA cores (rule R1:
+// IEEE FMA only, never tensor cores) in the frozen prefill order (V=1, L=1, P=1): every output is one
+// accumulation chain per K segment, strictly ascending in k; segments are summed in ascending order and
+// the bias comes last (rule R3).
+//
+// One packed fma.rn.f32x2 advances the chains of two neighbouring output columns (n, n+1) of the same row
+// by one element; each half is an ordinary fma.rn.f32, so the pairing is invisible in the bits.
+//
+// What bounds this loop on B200 (measured): a scheduler issues one instruction every other cycle while the
+// packed FMA, which occupies the pipe for two cycles, dominates, so every instruction that is not a packed
+// FMA costs an FMA slot.  The sustained fraction of the FP32 peak is therefore the share of packed FMAs in
+// the instruction stream, and the schedule below exists to keep everything else out of it:
+//   * 8 x 8 outputs per thread: four 16-byte shared loads per 32 packed FMAs;
+//   * a thread wants its eight activations of one k in two 16-byte loads, which needs the tile k-major in
+//     shared memory.  A small first kernel transposes x into a workspace xT [K][M]; TMA brings tiles
+//     [32 k][16 TR rows] of it to shared memory.  No thread spends registers, loads, stores, address
+//     arithmetic or bounds checks on staging activations, and the multiply loop keeps few values live (the
+//     128-register budget of two blocks per SM otherwise forces the compiler to recompute addresses);
+//   * the weight tile arrives by TMA too, in its stored 16-bit format; it has to become FP32 (Eq. 2: the
+//     upcast is exact) and k-major, so that one 16-byte load yields two (n, n+1) operand pairs.  Each thread
+//     converts 16 weights per slab: one 16-byte shared load, eight widenings and eight stores, twice.  TMA
+//     fills out-of-range rows and columns with zeros, so there are no bounds checks;
+//   * all shared-memory offsets of the multiply loop are immediates (the loop over a slab is unrolled).
+// Schedule (numerically inert): 256 threads, block tile 16 TR rows x 128 columns (TR = 5 .. 8 rows per
+// thread, whichever pads the batch least), two blocks per SM, K walked in slabs of 32; three activation
+// stages, two raw weight stages, two converted weight buffers.  One block-wide barrier per slab orders the
+// converted buffers and frees the stages that were just read, which one thread then refills through TMA.
+//
+// Every wait on a TMA completion is bounded: a wait that expires records the fact in the device status
+// word and the block returns without storing.
+#include "internal.h"
+#include "device_utils.cuh"
+#include "pipeline_utils.cuh"
+
+namespace detlin {
+
+namespace {
+
+using namespace pipe;
+
+constexpr int BN = 128, BK = 32;
+constexpr int kThreads = 256;
+constexpr int kXStages = 3;                          // activation ring
+constexpr int kRawBytes = BN * BK * 2;               // raw weight stage: [128 rows][32 k] 16-bit, 64-byte rows
+constexpr int kWfBytes = BK * BN * 4;                // converted weight buffer: [32 k][128 n] FP32, columns swizzled
+
+template <int TR> struct Tile {
+    static constexpr int BM = 16 * TR;
+    static constexpr int kXBytes = BK * BM * 4;      // [32 k][BM rows] FP32
+    // stages and buffers, then barriers and the abort word; 128 bytes of slack to align the first stage
+    static constexpr int kSmemBytes = kXStages * kXBytes + 2 * kRawBytes + 2 * kWfBytes + 128 + 128;
+};
+
+__device__ __forceinline__ void sts32(uint32_t addr, float v)
+{
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+// n consecutive floats from shared memory (n <= 4; the address is 4 n-byte aligned for n = 1, 2, 4)
+template <int N_>
+__device__ __forceinline__ void lds_floats(uint32_t addr, float* v)
+{
+    if constexpr (N_ == 4) {
+        const float4 t = lds128(addr);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else if constexpr (N_ == 2) {
+        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v[0]), "=f"(v[1]) : "r"(addr));
+    } else {
+#pragma unroll
+        for (int i = 0; i < N_; ++i) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v[i]) : "r"(addr + 4 * i));
+    }
+}
+__device__ __forceinline__ uint4 lds128u(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+template <int WF, int TR>
+__global__ void __launch_bounds__(kThreads, 2)
+prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                   const float* __restrict__ bias, float* __restrict__ out, int M, int N, int K, int seg_len, int direct,
+                   int tiles_m, int tiles_n, long long ldy, DeviceStatus* status, unsigned long long wait_limit_ns)
+{
+    typedef Tile<TR> T;
+    constexpr int TB = TR - 4;                       // rows of a thread in the upper group (1 .. 4)
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t xring = (smem_u32(smem_raw) + 127u) & ~127u;
+    const uint32_t raw0 = xring + kXStages * T::kXBytes;
+    const uint32_t wf0 = raw0 + 2 * kRawBytes;
+    const uint32_t xfull0 = wf0 + 2 * kWfBytes;
+    const uint32_t wfull0 = xfull0 + 8 * kXStages;
+    const uint32_t abort_flag = wfull0 + 8 * 2;
+
+    const int tid = threadIdx.x;
+    // 16 x 16 threads; a warp = 16 column groups x 2 row groups
+    const int tx = tid & 15, ty = tid >> 4;
+
+    // block -> (m tile fastest, then n tile, then segment)
+    long long u = blockIdx.x;
+    const int tm = (int)(u % tiles_m);
+    u /= tiles_m;
+    const int tn = (int)(u % tiles_n);
+    const int s = (int)(u / tiles_n);
+    const int m0 = tm * T::BM, n0 = tn * BN;
+    const int k_lo = s * seg_len;
+    const int k_hi = min(K, k_lo + seg_len);
+    const int n_slabs = (k_hi - k_lo + BK - 1) / BK;
+
+    if (tid == 0) {
+        for (int i = 0; i < kXStages; ++i) mbar_init(xfull0 + 8 * i, 1);
+        for (int i = 0; i < 2; ++i) mbar_init(wfull0 + 8 * i, 1);
+        sts_volatile_i32(abort_flag, 0);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    auto fill_x = [&](int slab) {                     // one thread: the activation tile of a slab into its stage
+        const int st = slab % kXStages;
+        mbar_arrive_expect_tx(xfull0 + 8 * st, T::kXBytes);
+        tma_load_2d_plain(xring + (uint32_t)st * T::kXBytes, &map_x, m0, k_lo + slab * BK, xfull0 + 8 * st);
+    };
+    auto fill_w = [&](int slab) {                     // one thread: the raw weight tile of a slab into its stage
+        const int st = slab & 1;
+        mbar_arrive_expect_tx(wfull0 + 8 * st, kRawBytes);
+        tma_load_2d_plain(raw0 + (uint32_t)st * kRawBytes, &map_w, k_lo + slab * BK, n0, wfull0 + 8 * st);
+    };
+    if (tid == 0) {
+        for (int i = 0; i < kXStages && i < n_slabs; ++i) fill_x(i);
+        for (int i = 0; i < 2 && i < n_slabs; ++i) fill_w(i);
+    }
+
+    // ---- conversion of a raw weight stage.  Piece p = tid + 256 j (j = 0, 1): row r = p >> 2, octet c = p & 3: the
+    //   eight lanes of a load phase read 128 contiguous bytes.  Weight (r, k = 8 c + e) goes to k row 8 c + e of
+    //   the converted buffer; inside a k row the 16-byte column group g = r >> 2 is stored at g ^ 2 c, which makes
+    //   the 32 lanes of a store (8 rows x 4 octets) hit 32 different banks.  The multiply loop reads whole
+    //   groups at one k, so the swizzle costs it one exclusive-or per octet.
+    uint32_t cv_src[2], cv_dst[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const int p = tid + 256 * j, r = p >> 2, c = p & 3;
+        cv_src[j] = (uint32_t)(r * 64 + c * 16);
+        cv_dst[j] = (uint32_t)((8 * c) * BN + ((((r >> 2) ^ (2 * c)) << 2) | (r & 3))) * 4u;
+    }
+    auto convert = [&](int slab) -> bool {
+        const int st = slab & 1;
+        if (!mbar_wait(wfull0 + 8 * st, (uint32_t)(slab >> 1) & 1u, abort_flag, status, wait_limit_ns, 3)) return false;
+        const uint32_t src = raw0 + (uint32_t)st * kRawBytes, dst = wf0 + (uint32_t)st * kWfBytes;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const uint4 v = lds128u(src + cv_src[j]);
+            const uint32_t a = dst + cv_dst[j];
+            sts32(a, up16_lo<WF>(v.x));
+            sts32(a + 1 * BN * 4, up16_hi<WF>(v.x));
+            sts32(a + 2 * BN * 4, up16_lo<WF>(v.y));
+            sts32(a + 3 * BN * 4, up16_hi<WF>(v.y));
+            sts32(a + 4 * BN * 4, up16_lo<WF>(v.z));
+            sts32(a + 5 * BN * 4, up16_hi<WF>(v.z));
+            sts32(a + 6 * BN * 4, up16_lo<WF>(v.w));
+            sts32(a + 7 * BN * 4, up16_hi<WF>(v.w));
+        }
+        return true;
+    };
+
+    // acc[i][j]: rows m0 + (i < 4 ? 4 ty + i : 64 + TB ty + i - 4); column pair j:
+    //   (n0 + 4 tx + 2 j, +1) for j < 2, (n0 + 64 + 4 tx + 2 (j - 2), +1) for j >= 2
+    float2 acc[TR][4];
+#pragma unroll
+    for (int i = 0; i < TR; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
+
+    // byte offsets of this thread's two row groups inside a k row of an activation stage
+    const uint32_t x_lo = (uint32_t)(4 * ty) * 4u, x_hi = (uint32_t)(64 + TB * ty) * 4u;
+
+    bool ok = convert(0);
+    if (!__syncthreads_and(ok)) return;
+    if (tid == 0 && 2 < n_slabs) fill_w(2);
+
+    for (int slab = 0; slab < n_slabs; ++slab) {
+        const int st = slab % kXStages;
+        if (slab + 1 < n_slabs) ok = convert(slab + 1);
+        if (ok) ok = mbar_wait(xfull0 + 8 * st, (uint32_t)(slab / kXStages) & 1u, abort_flag, status, wait_limit_ns, 4);
+
+        const uint32_t xs = xring + (uint32_t)st * T::kXBytes;
+        const uint32_t wb = wf0 + (uint32_t)(slab & 1) * kWfBytes;
+        // k beyond the end of the segment is skipped, not zero-filled; segments end on multiples of 8
+        const int n_oct = ok ? (min(BK, k_hi - (k_lo + slab * BK)) >> 3) : 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (c < n_oct) {
+                const uint32_t wc = wb + (uint32_t)(8 * c * BN) * 4u + (uint32_t)((tx ^ (2 * c)) << 4);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {        // k = 8 c + e
+                    const uint32_t xk = xs + (uint32_t)((8 * c + e) * T::BM) * 4u;
+                    float xv[TR];
+                    lds_floats<4>(xk + x_lo, xv);
+                    lds_floats<TB>(xk + x_hi, xv + 4);
+                    const float4 wa = lds128(wc + (uint32_t)(e * BN) * 4u);
+                    const float4 wd = lds128(wc + (uint32_t)(e * BN + 64) * 4u);
+                    const float2 wp[4] = {make_float2(wa.x, wa.y), make_float2(wa.z, wa.w), make_float2(wd.x, wd.y),
+                                          make_float2(wd.z, wd.w)};
+                    // column pair outermost: consecutive instructions share the weight operand (measured faster)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int i = 0; i < TR; ++i) acc[i][j] = __ffma2_rn(make_float2(xv[i], xv[i]), wp[j], acc[i][j]);
+                }
+            }
+        }
+        // the barrier carries the vote: a wait that expired anywhere in the block ends the block, nobody stores
+        if (!__syncthreads_and(ok)) return;
+        // every thread has finished reading this slab's activation stage and the raw stage of the next slab
+        if (tid == 0) {
+            if (slab + kXStages < n_slabs) fill_x(slab + kXStages);
+            if (slab + 3 < n_slabs) fill_w(slab + 3);
+        }
+    }
+
+    // ---- epilogue: bias (direct) or the segment's partial ----
+    const bool vec_ok = direct ? (ldy % 4 == 0) : (N % 4 == 0);     // rows of the destination start 16-byte aligned
+#pragma unroll
+    for (int i = 0; i < TR; ++i) {
+        const int m = m0 + (i < 4 ? 4 * ty + i : 64 + TB * ty + (i - 4));
+        if (m >= M) continue;
+        float* orow = direct ? out + (long long)m * ldy : out + ((long long)s * M + m) * N;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int n = n0 + 64 * h + 4 * tx;
+            float v[4] = {acc[i][2 * h].x, acc[i][2 * h].y, acc[i][2 * h + 1].x, acc[i][2 * h + 1].y};
+            if (direct && bias) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (n + e < N) v[e] = __fadd_rn(v[e], bias[n + e]);
+            }
+            if (vec_ok && n + 3 < N) {
+                *reinterpret_cast<float4*>(orow + n) = make_float4(v[0], v[1], v[2], v[3]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (n + e < N) orow[n + e] = v[e];
+            }
+        }
+    }
+}
+
+// First pass: xT[k][m] = x[m][k] for m < M, 0 for M <= m < ldt (ldt = M rounded up to a multiple of 4, the row pitch
+// of xT).  32 x 32 tiles through shared memory: reads and writes are both 128-byte rows.
+__global__ void __launch_bounds__(256) transpose_x_kernel(const float* __restrict__ x, float* __restrict__ xT, int M, int K, int ldt)
+{
+    __shared__ float tile[32][33];
+    const int k0 = blockIdx.x * 32, m0 = blockIdx.y * 32;
+    const int c = threadIdx.x & 31, r0 = threadIdx.x >> 5;
+#pragma unroll
+    for (int r = r0; r < 32; r += 8) {
+        const int m = m0 + r, k = k0 + c;
+        tile[r][c] = (m < M && k < K) ? x[(long long)m * K + k] : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = r0; r < 32; r += 8) {
+        const int k = k0 + r, m = m0 + c;
+        if (k < K && m < ldt) xT[(long long)k * ldt + m] = tile[c][r];
+    }
+}
+
+template <int WF, int TR>
+cudaError_t launch_t(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
+{
+    typedef Tile<TR> T;
+    static bool configured[kMaxDevices];             // function attributes belong to a device
+    int dev = 0;
+    cudaError_t de = cudaGetDevice(&dev);
+    if (de != cudaSuccess) return de;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_tma_kernel<WF, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    const int tiles_m = (int)((a.M + T::BM - 1) / T::BM), tiles_n = (int)((a.N + BN - 1) / BN);
+    const long long units = (long long)tiles_m * tiles_n * a.S;
+    if (units > 0x7fffffffLL) return cudaErrorInvalidValue;
+    const int direct = (a.S == 1);
+    prefill_tma_kernel<WF, TR><<<(unsigned)units, kThreads, T::kSmemBytes, a.stream>>>(
+        *map_x, *map_w, a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N, (int)a.K, (int)a.seg_len, direct, tiles_m, tiles_n,
+        (long long)a.ldy, a.status, a.wait_limit_ns);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (!direct) return launch_combine(a);
+    return cudaSuccess;
+}
+
+template <int WF>
+cudaError_t launch_f(const LaunchArgs& a, int tr, const CUtensorMap* map_w, const CUtensorMap* map_x)
+{
+    switch (tr) {
+    case 5: return launch_t<WF, 5>(a, map_w, map_x);
+    case 6: return launch_t<WF, 6>(a, map_w, map_x);
+    case 7: return launch_t<WF, 7>(a, map_w, map_x);
+    default: return launch_t<WF, 8>(a, map_w, map_x);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_transpose_x(const float* x, float* xT, int64_t M, int64_t K, int64_t ldt, cudaStream_t stream)
+{
+    const long long by = (ldt + 31) / 32, bx = (K + 31) / 32;
+    dim3 grid((unsigned)bx, 1);
+    // grid.y carries the rows (at most 65535 blocks per launch): larger M is cut into slabs of rows
+    for (long long y0 = 0; y0 < by; y0 += 32768) {
+        grid.y = (unsigned)((by - y0 < 32768) ? by - y0 : 32768);
+        const long long m0 = y0 * 32;
+        transpose_x_kernel<<<grid, 256, 0, stream>>>(x + m0 * K, xT + m0, (int)(M - m0), (int)K, (int)ldt);
+    }
+    return cudaGetLastError();
+}
+
+// Tensor maps the caller builds, both without swizzle: the transposed activations xT [K][ldt] FP32 with box
+// [32][16 tr]; W [N][K] 16-bit with box [128][32].
+cudaError_t launch_prefill_tma(const LaunchArgs& a, int tr, const CUtensorMap* map_w, const CUtensorMap* map_x)
+{
+    if (!a.status) return cudaErrorInvalidValue;
+    switch (a.wfmt) {
+    case DET_WEIGHT_BF16: return launch_f<0>(a, tr, map_w, map_x);
+    case DET_WEIGHT_FP16: return launch_f<1>(a, tr, map_w, map_x);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace detlin

@@ -195,7 +195,8 @@ def test_prefill_tile_heights_bit_exact(M, N, K):
     sizes just above a multiple of 128 get a shorter tile)."""
     x, W, b = inputs.make_case(M, N, K)
     want = oracle_y(x, W, b)
-    for variant in (0, 5, 6, 7, 8):
+    # 5 .. 8: the TMA-fed kernel with that many rows per thread; 15 .. 18: the register-staged kernel
+    for variant in (0, 5, 6, 7, 8, 15, 16, 17, 18):
         assert_bits_equal(run_gpu(x, W, b, kernel=KERNEL_PREFILL, variant=variant), want, f"rows per thread {variant}")
 
 
