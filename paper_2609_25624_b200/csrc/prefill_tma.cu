@@ -22,8 +22,8 @@
 //     fills out-of-range rows and columns with zeros, so there are no bounds checks;
 //   * all shared-memory offsets of the multiply loop are immediates (the loop over a slab is unrolled).
 // Schedule (numerically inert): 256 threads, block tile 16 TR rows x 128 columns (TR = 5 .. 8 rows per
-// thread, whichever pads the batch least), two blocks per SM, K walked in slabs of 32; three activation
-// stages, two raw weight stages, two converted weight buffers.  One block-wide barrier per slab orders the
+// thread, whichever pads the batch least), two blocks per SM, K walked in slabs of 32; two activation
+// stages, two raw weight stages, two converted weight buffers, all indexed by the parity of the slab.  One block-wide barrier per slab orders the
 // converted buffers and frees the stages that were just read, which one thread then refills through TMA.
 //
 // Every wait on a TMA completion is bounded: a wait that expires records the fact in the device status
@@ -31,6 +31,7 @@
 #include "internal.h"
 #include "device_utils.cuh"
 #include "pipeline_utils.cuh"
+#include <type_traits>
 
 namespace detlin {
 
@@ -40,7 +41,7 @@ using namespace pipe;
 
 constexpr int BN = 128, BK = 32;
 constexpr int kThreads = 256;
-constexpr int kXStages = 3;                          // activation ring
+constexpr int kXStages = 2;                          // activation stages (slab parity)
 constexpr int kRawBytes = BN * BK * 2;               // raw weight stage: [128 rows][32 k] 16-bit, 64-byte rows
 constexpr int kWfBytes = BK * BN * 4;                // converted weight buffer: [32 k][128 n] FP32, columns swizzled
 
@@ -141,14 +142,16 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         cv_src[j] = (uint32_t)(r * 64 + c * 16);
         cv_dst[j] = (uint32_t)((8 * c) * BN + ((((r >> 2) ^ (2 * c)) << 2) | (r & 3))) * 4u;
     }
-    auto convert = [&](int slab) -> bool {
-        const int st = slab & 1;
-        if (!mbar_wait(wfull0 + 8 * st, (uint32_t)(slab >> 1) & 1u, abort_flag, status, wait_limit_ns, 3)) return false;
-        const uint32_t src = raw0 + (uint32_t)st * kRawBytes, dst = wf0 + (uint32_t)st * kWfBytes;
+    // Slabs alternate between two sets of buffers; the parity P of a slab is a compile-time constant of the code
+    // that handles it (the slab loop is unrolled by two), so every shared-memory address of the multiply loop is a
+    // per-thread base plus an immediate.
+    auto convert = [&](int slab, auto par) -> bool {
+        constexpr int P = decltype(par)::value;
+        if (!mbar_wait(wfull0 + 8 * P, (uint32_t)(slab >> 1) & 1u, abort_flag, status, wait_limit_ns, 3)) return false;
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-            const uint4 v = lds128u(src + cv_src[j]);
-            const uint32_t a = dst + cv_dst[j];
+            const uint4 v = lds128u(raw0 + P * kRawBytes + cv_src[j]);
+            const uint32_t a = wf0 + P * kWfBytes + cv_dst[j];
             sts32(a, up16_lo<WF>(v.x));
             sts32(a + 1 * BN * 4, up16_hi<WF>(v.x));
             sts32(a + 2 * BN * 4, up16_lo<WF>(v.y));
@@ -169,51 +172,66 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
 
-    // byte offsets of this thread's two row groups inside a k row of an activation stage
-    const uint32_t x_lo = (uint32_t)(4 * ty) * 4u, x_hi = (uint32_t)(64 + TB * ty) * 4u;
+    // this thread's two row groups inside a k row of an activation stage, and its column group inside a k row
+    // of a converted weight buffer for each octet of k (the swizzle of the conversion)
+    const uint32_t x_lo = xring + (uint32_t)(4 * ty) * 4u, x_hi = xring + (uint32_t)(64 + TB * ty) * 4u;
+    uint32_t w_oct[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) w_oct[c] = wf0 + (uint32_t)(8 * c * BN) * 4u + (uint32_t)((tx ^ (2 * c)) << 4);
 
-    bool ok = convert(0);
-    if (!__syncthreads_and(ok)) return;
-    if (tid == 0 && 2 < n_slabs) fill_w(2);
+    // one octet of k: k = 8 c + e inside the slab
+    auto octet = [&](uint32_t xlo, uint32_t xhi, uint32_t wc) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float xv[TR];
+            lds_floats<4>(xlo + (uint32_t)(e * T::BM) * 4u, xv);
+            lds_floats<TB>(xhi + (uint32_t)(e * T::BM) * 4u, xv + 4);
+            const float4 wa = lds128(wc + (uint32_t)(e * BN) * 4u);
+            const float4 wd = lds128(wc + (uint32_t)(e * BN + 64) * 4u);
+            const float2 wp[4] = {make_float2(wa.x, wa.y), make_float2(wa.z, wa.w), make_float2(wd.x, wd.y),
+                                  make_float2(wd.z, wd.w)};
+            // column pair outermost: consecutive instructions share the weight operand (measured faster)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int i = 0; i < TR; ++i) acc[i][j] = __ffma2_rn(make_float2(xv[i], xv[i]), wp[j], acc[i][j]);
+        }
+    };
 
-    for (int slab = 0; slab < n_slabs; ++slab) {
-        const int st = slab % kXStages;
-        if (slab + 1 < n_slabs) ok = convert(slab + 1);
-        if (ok) ok = mbar_wait(xfull0 + 8 * st, (uint32_t)(slab / kXStages) & 1u, abort_flag, status, wait_limit_ns, 4);
-
-        const uint32_t xs = xring + (uint32_t)st * T::kXBytes;
-        const uint32_t wb = wf0 + (uint32_t)(slab & 1) * kWfBytes;
+    // one slab of parity P; returns false when a wait expired somewhere in the block (then nobody stores)
+    auto do_slab = [&](int slab, auto par) -> bool {
+        constexpr int P = decltype(par)::value;
+        bool ok = true;
+        if (slab + 1 < n_slabs) ok = convert(slab + 1, std::integral_constant<int, P ^ 1>());
+        if (ok) ok = mbar_wait(xfull0 + 8 * P, (uint32_t)(slab >> 1) & 1u, abort_flag, status, wait_limit_ns, 4);
         // k beyond the end of the segment is skipped, not zero-filled; segments end on multiples of 8
         const int n_oct = ok ? (min(BK, k_hi - (k_lo + slab * BK)) >> 3) : 0;
+        if (n_oct == 4) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if (c < n_oct) {
-                const uint32_t wc = wb + (uint32_t)(8 * c * BN) * 4u + (uint32_t)((tx ^ (2 * c)) << 4);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {        // k = 8 c + e
-                    const uint32_t xk = xs + (uint32_t)((8 * c + e) * T::BM) * 4u;
-                    float xv[TR];
-                    lds_floats<4>(xk + x_lo, xv);
-                    lds_floats<TB>(xk + x_hi, xv + 4);
-                    const float4 wa = lds128(wc + (uint32_t)(e * BN) * 4u);
-                    const float4 wd = lds128(wc + (uint32_t)(e * BN + 64) * 4u);
-                    const float2 wp[4] = {make_float2(wa.x, wa.y), make_float2(wa.z, wa.w), make_float2(wd.x, wd.y),
-                                          make_float2(wd.z, wd.w)};
-                    // column pair outermost: consecutive instructions share the weight operand (measured faster)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-#pragma unroll
-                        for (int i = 0; i < TR; ++i) acc[i][j] = __ffma2_rn(make_float2(xv[i], xv[i]), wp[j], acc[i][j]);
-                }
-            }
+            for (int c = 0; c < 4; ++c)
+                octet(x_lo + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u, x_hi + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u,
+                      w_oct[c] + P * kWfBytes);
+        } else {
+#pragma unroll 1
+            for (int c = 0; c < n_oct; ++c)
+                octet(x_lo + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u, x_hi + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u,
+                      wf0 + P * kWfBytes + (uint32_t)(8 * c * BN) * 4u + (uint32_t)((tx ^ (2 * c)) << 4));
         }
-        // the barrier carries the vote: a wait that expired anywhere in the block ends the block, nobody stores
-        if (!__syncthreads_and(ok)) return;
+        // the barrier carries the vote
+        if (!__syncthreads_and(ok)) return false;
         // every thread has finished reading this slab's activation stage and the raw stage of the next slab
         if (tid == 0) {
-            if (slab + kXStages < n_slabs) fill_x(slab + kXStages);
+            if (slab + 2 < n_slabs) fill_x(slab + 2);
             if (slab + 3 < n_slabs) fill_w(slab + 3);
         }
+        return true;
+    };
+
+    if (!__syncthreads_and(convert(0, std::integral_constant<int, 0>()))) return;
+    if (tid == 0 && 2 < n_slabs) fill_w(2);
+    for (int slab = 0; slab < n_slabs; slab += 2) {
+        if (!do_slab(slab, std::integral_constant<int, 0>())) return;
+        if (slab + 1 < n_slabs && !do_slab(slab + 1, std::integral_constant<int, 1>())) return;
     }
 
     // ---- epilogue: bias (direct) or the segment's partial ----
