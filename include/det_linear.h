@@ -91,6 +91,10 @@ DET_API det_status_t det_linear_plan_params(int64_t M, int64_t N, int64_t K, det
  * status word and, in the prefill bucket when S > 1, the split-K partials workspace (device); the
  * decode bucket folds its segments inside the kernel and needs none.  Returns NULL on failure
  * (det_last_error(), det_last_status()).
+ * A prefill plan for 16-bit weights also asks for 4 * K * roundup(M, 4) bytes in which every run
+ * writes x transposed for its TMA-fed kernel (schedule only; reported as "activation_workspace_bytes"
+ * by det_linear_plan_describe, not in workspace_bytes).  If that allocation fails the plan is still
+ * created and runs the register-staged kernel, which computes the same bits.
  * A plan may be used from one stream at a time: its workspace is not re-entrant; make one plan
  * per stream for concurrent use.  Destroy with det_linear_plan_destroy.
  */
@@ -193,8 +197,9 @@ DET_API det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream
 DET_API det_status_t det_linear_plan_get_params(const det_linear_plan_t* plan, det_linear_params_t* out);
 
 /* Write a JSON description (bucket, V, L, P, S, seg_len, order_version, kernel, workspace_bytes, the shard
- * and, for the decode kernel, the tiling in use on the current device with its resident blocks per SM --
- * schedule only)
+ * and, schedule only: for the decode kernel the tiling in use on the current device with its resident
+ * blocks per SM, for the prefill kernel the tile, how it is fed ("tma" or "registers") and the bytes of
+ * the activation workspace)
  * to buf (at most n bytes including the terminator).  DET_ERR_INVALID_ARG if it does not fit. */
 DET_API det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, size_t n);
 

@@ -37,8 +37,9 @@ DET_API void det_test_fail_next_alloc(int nth);
 
 /*
  * Bound of one device-side wait for the kernels launched through this plan (default 2 s), and flags:
- * bit 0 (value 1) is a deliberate stall: thread block 0 of the decode kernel never
- * requests the activations of its first stage, so the wait for that stage runs into the bound.  The
+ * bit 0 (value 1) is a deliberate stall: thread block 0 of the decode kernel (of the TMA-fed prefill
+ * kernel likewise) never requests the activations of its first stage, so the wait for that stage runs
+ * into the bound.  The
  * kernel then records the timeout in the plan's status word, drains and returns (no trap, no endless
  * loop; the other blocks finish normally), and det_linear_plan_check reports DET_ERR_DEVICE_TIMEOUT.
  * The output of such a run is undefined.  Reset with (2000000000, 0).

@@ -227,8 +227,8 @@ def det_linear_plan_get_params(plan: Plan) -> Params:
 
 
 def det_linear_plan_describe(plan: Plan) -> dict:
-    buf = ctypes.create_string_buffer(512)
-    _check(lib().det_linear_plan_describe(plan.handle, buf, 512))
+    buf = ctypes.create_string_buffer(1024)
+    _check(lib().det_linear_plan_describe(plan.handle, buf, 1024))
     return json.loads(buf.value.decode())
 
 

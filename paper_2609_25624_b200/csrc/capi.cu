@@ -445,12 +445,14 @@ det_status_t det_linear_plan_describe(const det_linear_plan_t* plan, char* buf, 
                      "{\"mt\": %d, \"wm\": %d, \"rt\": %d, \"wr\": %d, \"sk\": %d, \"kc\": %d, \"stages\": %d, \"blocks_per_sm\": %d}",
                      c.mt, c.wm, c.rt, c.wr, c.sk, c.kc, c.stages, decode_config_occupancy(p.weight_format, c, p.S));
     }
-    char ptile[96] = "null";
+    char ptile[160] = "null";
     if (p.kernel == kKernelPrefill) {
         const int v = plan->variant;
         const bool staged = !plan->x_t || (v >= 15 && v <= 18);
         const int tr = (v >= 5 && v <= 8) ? v : (v >= 15 && v <= 18) ? v - 10 : prefill_rows_per_thread(p.M);
-        snprintf(ptile, sizeof ptile, "{\"bm\": %d, \"bn\": 128, \"bk\": 32, \"feed\": \"%s\"}", 16 * tr, staged ? "registers" : "tma");
+        snprintf(ptile, sizeof ptile, "{\"bm\": %d, \"bn\": 128, \"bk\": 32, \"feed\": \"%s\", \"activation_workspace_bytes\": %llu}",
+                 16 * tr, staged ? "registers" : "tma",
+                 plan->x_t ? 4ull * (unsigned long long)((p.M + 3) / 4 * 4) * (unsigned long long)p.K : 0ull);
     }
     int w = snprintf(buf, n,
                      "{\"M\": %lld, \"N\": %lld, \"K\": %lld, \"bucket\": \"%s\", \"V\": %d, \"L\": %d, \"P\": %d, "

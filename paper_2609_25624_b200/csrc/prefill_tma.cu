@@ -81,7 +81,8 @@ template <int WF, int TR>
 __global__ void __launch_bounds__(kThreads, 2)
 prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                    const float* __restrict__ bias, float* __restrict__ out, int M, int N, int K, int seg_len, int direct,
-                   int tiles_m, int tiles_n, long long ldy, DeviceStatus* status, unsigned long long wait_limit_ns)
+                   int tiles_m, int tiles_n, long long ldy, DeviceStatus* status, unsigned long long wait_limit_ns,
+                   int test_flags)
 {
     typedef Tile<TR> T;
     constexpr int TB = TR - 4;                       // rows of a thread in the upper group (1 .. 4)
@@ -126,7 +127,8 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         tma_load_2d_plain(raw0 + (uint32_t)st * kRawBytes, &map_w, k_lo + slab * BK, n0, wfull0 + 8 * st);
     };
     if (tid == 0) {
-        for (int i = 0; i < kXStages && i < n_slabs; ++i) fill_x(i);
+        // (test hook: block 0 never requests its first activation tile, so its first wait expires)
+        for (int i = ((test_flags & 1) && blockIdx.x == 0) ? 1 : 0; i < kXStages && i < n_slabs; ++i) fill_x(i);
         for (int i = 0; i < 2 && i < n_slabs; ++i) fill_w(i);
     }
 
@@ -301,7 +303,7 @@ cudaError_t launch_t(const LaunchArgs& a, const CUtensorMap* map_w, const CUtens
     const int direct = (a.S == 1);
     prefill_tma_kernel<WF, TR><<<(unsigned)units, kThreads, T::kSmemBytes, a.stream>>>(
         *map_x, *map_w, a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N, (int)a.K, (int)a.seg_len, direct, tiles_m, tiles_n,
-        (long long)a.ldy, a.status, a.wait_limit_ns);
+        (long long)a.ldy, a.status, a.wait_limit_ns, a.test_flags);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (!direct) return launch_combine(a);

@@ -98,3 +98,54 @@ def test_bounded_wait_expires_and_the_kernel_returns(M, N, K):
     B.det_linear_plan_check(plan)
     plan.close()
     assert_bits_equal(y.cpu().numpy(), want, "after the expired wait")
+
+
+def test_bounded_wait_expires_in_the_prefill_kernel():
+    """The TMA-fed prefill kernel bounds its waits too: block 0 is made to miss its first activation tile,
+    gives up after the limit and returns; the plan reports it and works again afterwards."""
+    M, N, K = 128, 256, 1024
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    xd, Wd, bd = x.cuda(), W.cuda(), b.cuda()
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    plan = B.det_linear_plan(M, N, K)
+    d = B.det_linear_plan_describe(plan)
+    assert d["kernel"] == "prefill" and d["prefill_tile"]["feed"] == "tma"
+    B.det_test_plan_set_wait(plan, 5_000_000, withhold_first_copy=True)     # 5 ms per wait
+    t0 = time.perf_counter()
+    B.det_linear_run(plan, xd, Wd, bd, y)
+    with pytest.raises(B.DetLinearError) as ei:
+        B.det_linear_plan_check(plan)
+    elapsed = time.perf_counter() - t0
+    assert ei.value.status == DET_ERR_DEVICE_TIMEOUT
+    assert "site 4" in B.det_last_error() or "site 3" in B.det_last_error()
+    assert elapsed < 5.0, f"the stalled kernel took {elapsed:.2f} s to give up"
+    B.det_test_plan_set_wait(plan, 2_000_000_000, withhold_first_copy=False)
+    y.fill_(float("nan"))
+    B.det_linear_run(plan, xd, Wd, bd, y)
+    B.det_linear_plan_check(plan)
+    plan.close()
+    assert_bits_equal(y.cpu().numpy(), want, "after the expired wait")
+
+
+@pytest.mark.parametrize("M,N,K,nth", [(128, 256, 4096, 3), (96, 136, 256, 2)])
+def test_prefill_without_its_activation_workspace(M, N, K, nth):
+    """The transposed-activation workspace is optional: when its allocation fails the plan is still created,
+    runs the register-staged kernel and produces the same bits."""
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    assert (B.det_linear_plan_params(M, N, K).workspace_bytes > 0) == (nth == 3)
+    B.det_test_fail_next_alloc(nth)                 # status word, (partials,) then the workspace
+    try:
+        plan = B.det_linear_plan(M, N, K)
+    finally:
+        B.det_test_fail_next_alloc(0)
+    assert B.det_linear_plan_describe(plan)["prefill_tile"]["feed"] == "registers"
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    B.det_linear_run(plan, x.cuda(), W.cuda(), b.cuda(), y)
+    B.det_linear_plan_check(plan)
+    plan.close()
+    assert_bits_equal(y.cpu().numpy(), want, "register-staged fallback")
+    plan = B.det_linear_plan(M, N, K)
+    assert B.det_linear_plan_describe(plan)["prefill_tile"]["feed"] == "tma"
+    plan.close()
