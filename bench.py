@@ -424,6 +424,7 @@ def calibration(B, dev, fp32_peak):
     out = {"fp32_peak_derived_tflops": fp32_peak,
            "fp32_fma_measured_tflops": B.det_test_measure_fma_peak(False),
            "fp32_fma2_measured_tflops": B.det_test_measure_fma_peak(True),
+           "fp32_prefill_loop_alone_tflops": B.det_test_measure_fma_peak(2),
            "hbm_read_only_measured_gbs": B.det_test_measure_read_bandwidth(buf)}
     del buf
     return out

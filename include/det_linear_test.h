@@ -60,7 +60,9 @@ DET_API void det_test_green_stream_destroy(void* handle);
 /*
  * Calibration for the benchmark's rooflines (these compute nothing of the method).
  * det_test_measure_fma_peak: FP32 multiply-add issue peak of the CUDA cores in TFLOP/s, measured
- * with a register-only loop of scalar fma.rn.f32 (packed = 0) or fma.rn.f32x2 (packed = 1).
+ * with a register-only loop of scalar fma.rn.f32 (packed = 0) or fma.rn.f32x2 (packed = 1); packed = 2
+ * times the prefill kernel's multiply loop alone (8 x 8 outputs per thread from resident shared-memory tiles,
+ * no staging, no barriers): the ceiling of that loop.
  * det_test_measure_read_bandwidth: read-only streaming rate in GB/s over `bytes` of device memory
  * at `buf` (16-byte aligned, at least 1 MiB; use a buffer much larger than L2).
  * Both run on the default stream and synchronise.

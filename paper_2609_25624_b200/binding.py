@@ -377,10 +377,11 @@ def det_test_green_stream_destroy(handle) -> None:
     lib().det_test_green_stream_destroy(handle)
 
 
-def det_test_measure_fma_peak(packed: bool) -> float:
-    """Measured FP32 FMA issue peak of the CUDA cores in TFLOP/s (scalar or packed FP32x2)."""
+def det_test_measure_fma_peak(packed) -> float:
+    """Measured FP32 FMA issue peak of the CUDA cores in TFLOP/s: False/0 scalar, True/1 packed FP32x2,
+    2 the prefill multiply loop alone on resident shared-memory tiles."""
     out = ctypes.c_double(0.0)
-    _check(lib().det_test_measure_fma_peak(1 if packed else 0, ctypes.byref(out)))
+    _check(lib().det_test_measure_fma_peak(int(packed), ctypes.byref(out)))
     return out.value
 
 

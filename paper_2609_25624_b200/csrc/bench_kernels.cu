@@ -35,6 +35,47 @@ __global__ void __launch_bounds__(256) fma_peak_kernel(float* out, int iters)
     if (r == 123.456f) out[0] = r;    // keeps the loop alive without a store on the normal path
 }
 
+// The prefill multiply loop alone: 8 x 8 outputs per thread, both operand tiles k-major and resident in shared
+// memory, four 16-byte loads per 32 packed FMAs, no staging, no barriers: the ceiling of that loop.
+__global__ void __launch_bounds__(256, 2) fma_loop_kernel(float* out, int iters, const float* __restrict__ in)
+{
+    __shared__ __align__(16) float tile[2 * 32 * 132];
+    for (int i = threadIdx.x; i < 2 * 32 * 132; i += 256) tile[i] = in[i & 63];
+    __syncthreads();
+    const uint32_t base = (uint32_t)__cvta_generic_to_shared(tile);
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const uint32_t xb = base + ty * 16, xb2 = xb + 64 * 4, wb = base + 32 * 132 * 4 + tx * 16;
+    float2 acc[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int p = 0; p < 4; ++p) acc[i][p] = make_float2((float)i, (float)p);
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll 8
+        for (int kk = 0; kk < 32; ++kk) {
+            float4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t a = (q == 0 ? xb : q == 1 ? xb2 : q == 2 ? wb : wb + 64 * 4) + kk * 132 * 4;
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v[q].x), "=f"(v[q].y), "=f"(v[q].z), "=f"(v[q].w) : "r"(a));
+            }
+            const float xv[8] = {v[0].x, v[0].y, v[0].z, v[0].w, v[1].x, v[1].y, v[1].z, v[1].w};
+            const float2 wp[4] = {make_float2(v[2].x, v[2].y), make_float2(v[2].z, v[2].w), make_float2(v[3].x, v[3].y),
+                                  make_float2(v[3].z, v[3].w)};
+#pragma unroll
+            for (int p = 0; p < 4; ++p)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[i][p] = __ffma2_rn(make_float2(xv[i], xv[i]), wp[p], acc[i][p]);
+        }
+    }
+    float r = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int p = 0; p < 4; ++p) r += acc[i][p].x + acc[i][p].y;
+    if (r == 123.456f) out[0] = r;
+}
+
 __global__ void __launch_bounds__(512) read_stream_kernel(const uint4* __restrict__ p, size_t n, unsigned* out)
 {
     unsigned acc = 0;
@@ -79,15 +120,18 @@ det_status_t det_test_measure_fma_peak(int packed, double* tflops_out)
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     float* out = nullptr;
     if (e == cudaSuccess) e = cudaMalloc(&out, 256);
+    if (e == cudaSuccess) e = cudaMemset(out, 0, 256);
     if (e != cudaSuccess) { set_error("measure_fma_peak: %s", cudaGetErrorString(e)); return DET_ERR_CUDA; }
-    const int iters = 4096, blocks = sms * 8;
+    const bool loop = (packed == 2);                 // the prefill multiply loop on resident shared memory
+    const int iters = loop ? 2048 : 4096, blocks = loop ? sms * 2 : sms * 8;
     cudaEvent_t e0, e1;
     cudaEventCreate(&e0);
     cudaEventCreate(&e1);
     float best = 1e30f;
     for (int rep = 0; rep < 6; ++rep) {
         cudaEventRecord(e0);
-        if (packed) fma_peak_kernel<1><<<blocks, 256>>>(out, iters);
+        if (loop) fma_loop_kernel<<<blocks, 256>>>(out, iters, out);
+        else if (packed) fma_peak_kernel<1><<<blocks, 256>>>(out, iters);
         else        fma_peak_kernel<0><<<blocks, 256>>>(out, iters);
         cudaEventRecord(e1);
         e = cudaEventSynchronize(e1);
@@ -100,8 +144,8 @@ det_status_t det_test_measure_fma_peak(int packed, double* tflops_out)
     cudaEventDestroy(e1);
     cudaFree(out);
     if (e != cudaSuccess) { set_error("measure_fma_peak: %s", cudaGetErrorString(e)); return DET_ERR_CUDA; }
-    // per thread and iteration: 4 x 16 x 2 FMAs = 256 flop
-    *tflops_out = 256.0 * iters * 256.0 * blocks / (best * 1e-3) / 1e12;
+    // per thread and iteration: 4 x 16 x 2 FMAs = 256 flop (register loops); 32 k x 64 FMAs = 4096 flop (tile loop)
+    *tflops_out = (loop ? 4096.0 : 256.0) * iters * 256.0 * blocks / (best * 1e-3) / 1e12;
     return DET_OK;
 }
 
