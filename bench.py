@@ -640,7 +640,7 @@ def attention_table(B, dev, st, hbm_peak):
         reps = 4
         ms = time_graph(lambda: [B.det_attention_decode(q, k, v, scale, o) for _ in range(reps)], 3, st) / reps
         nbytes = 8 * Bt * Hkv * T * D + 8 * Bt * Hq * D
-        rows.append({"B": Bt, "Hq": Hq, "Hkv": Hkv, "T": T, "D": D, "blocks": Bt * Hkv, "us": ms * 1e3,
+        rows.append({"B": Bt, "Hq": Hq, "Hkv": Hkv, "T": T, "D": D, "rows": Bt * Hkv, "us": ms * 1e3,
                      "gbs": nbytes / ms / 1e6, "pct_hbm": 100 * nbytes / ms / 1e6 / hbm_peak,
                      "l2_resident": nbytes < (100 << 20)})
     return rows

@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.det_last_error.restype = ctypes.c_char_p
         L.det_order_version.restype = i32
         L.det_last_status.restype = i32
+        L.det_test_attention_set_split.argtypes = [i32]
+        L.det_test_attention_set_split.restype = None
         L.det_test_fail_next_alloc.argtypes = [i32]
         L.det_test_fail_next_alloc.restype = None
         L.det_test_plan_set_wait.argtypes = [p, ctypes.c_uint64, i32]
@@ -353,6 +355,11 @@ def det_test_plan_set_max_blocks(plan: Plan, max_blocks: int) -> None:
 
 def det_test_plan_set_variant(plan: Plan, variant: int) -> None:
     _check(lib().det_test_plan_set_variant(plan.handle, variant))
+
+
+def det_test_attention_set_split(blocks_per_row: int) -> None:
+    """Force the cluster size of det_attention_decode (1, 2, 4, 8; 0 = automatic).  Same bits for every value."""
+    lib().det_test_attention_set_split(blocks_per_row)
 
 
 def det_test_fail_next_alloc(nth: int = 1) -> None:

@@ -533,6 +533,8 @@ det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
     return DET_OK;
 }
 
+void det_test_attention_set_split(int blocks_per_row) { attention_test_force_split(blocks_per_row); }
+
 void det_test_fail_next_alloc(int nth)
 {
     g_fail_alloc_countdown = nth > 0 ? nth : 0;
