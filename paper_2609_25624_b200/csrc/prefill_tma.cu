@@ -265,7 +265,8 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 
 // First pass: xT[k][m] = x[m][k] for m < M, 0 for M <= m < ldt (ldt = M rounded up to a multiple of 4, the row pitch
 // of xT).  32 x 32 tiles through shared memory: reads and writes are both 128-byte rows.
-__global__ void __launch_bounds__(256) transpose_x_kernel(const float* __restrict__ x, float* __restrict__ xT, int M, int K, int ldt)
+// (x, xT, M and m_pad are those of the slab of rows this launch covers: m_pad = the slab's share of ldt.)
+__global__ void __launch_bounds__(256) transpose_x_kernel(const float* __restrict__ x, float* __restrict__ xT, int M, int m_pad, int K, int ldt)
 {
     __shared__ float tile[32][33];
     const int k0 = blockIdx.x * 32, m0 = blockIdx.y * 32;
@@ -279,7 +280,7 @@ __global__ void __launch_bounds__(256) transpose_x_kernel(const float* __restric
 #pragma unroll
     for (int r = r0; r < 32; r += 8) {
         const int k = k0 + r, m = m0 + c;
-        if (k < K && m < ldt) xT[(long long)k * ldt + m] = tile[c][r];
+        if (k < K && m < m_pad) xT[(long long)k * ldt + m] = tile[c][r];
     }
 }
 
@@ -331,7 +332,7 @@ cudaError_t launch_transpose_x(const float* x, float* xT, int64_t M, int64_t K, 
     for (long long y0 = 0; y0 < by; y0 += 32768) {
         grid.y = (unsigned)((by - y0 < 32768) ? by - y0 : 32768);
         const long long m0 = y0 * 32;
-        transpose_x_kernel<<<grid, 256, 0, stream>>>(x + m0 * K, xT + m0, (int)(M - m0), (int)K, (int)ldt);
+        transpose_x_kernel<<<grid, 256, 0, stream>>>(x + m0 * K, xT + m0, (int)(M - m0), (int)(ldt - m0), (int)K, (int)ldt);
     }
     return cudaGetLastError();
 }

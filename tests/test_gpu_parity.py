@@ -243,3 +243,17 @@ def test_plan_tune_changes_the_schedule_only():
     y = torch.empty(100, 256, device="cuda")
     assert B.det_linear_plan_tune(plan, x.cuda(), W.cuda(), b.cuda(), y) == (0, -1.0)
     plan.close()
+
+
+@pytest.mark.parametrize("M,N,K", [(70001, 24, 64), (1048700, 8, 32)])
+def test_prefill_very_tall_batches(M, N, K):
+    """Batches far taller than a grid dimension: the activation transpose walks the rows in slabs of 2^20 rows,
+    the multiply kernel numbers its tiles in one dimension.  Every element against the oracle."""
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    plan = B.det_linear_plan(M, N, K)
+    d = B.det_linear_plan_describe(plan)
+    assert d["kernel"] == "prefill" and d["prefill_tile"]["feed"] == "tma"
+    plan.close()
+    assert_bits_equal(run_gpu(x, W, b), want, "automatic")
+    assert_bits_equal(run_gpu(x, W, b, variant=18), want, "register-staged")
