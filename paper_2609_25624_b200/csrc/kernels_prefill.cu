@@ -6,8 +6,8 @@
 // One packed fma.rn.f32x2 advances the chains of two neighbouring output columns (n, n+1) of the
 // same row m by one element: operands (x[m,k], x[m,k]) and (up(W[n,k]), up(W[n+1,k])), accumulator
 // (acc[m,n], acc[m,n+1]).  Each half is an ordinary fma.rn.f32, so the pairing is invisible in the
-// bits.  Measured on B200 this loop sustains more than the scalar-FMA form of the same tile because
-// the packed instruction leaves every other issue slot free for the shared-memory loads.
+// bits.  Measured on B200 this loop sustains more than the scalar-FMA form of the same tile: the packed
+// instruction needs an issue slot every other cycle only.
 //
 // Schedule (numerically inert): 128 x 128 output tile per block (16 TR x 128 with TR = 5 .. 7 rows per
 // thread when that pads the batch less), 256 threads, 8 x 8 outputs per
