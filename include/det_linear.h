@@ -91,7 +91,7 @@ DET_API det_status_t det_linear_plan_params(int64_t M, int64_t N, int64_t K, det
  * status word and, in the prefill bucket when S > 1, the split-K partials workspace (device); the
  * decode bucket folds its segments inside the kernel and needs none.  Returns NULL on failure
  * (det_last_error(), det_last_status()).
- * A prefill plan for 16-bit weights also asks for 4 * K * roundup(M, 4) bytes in which every run
+ * A prefill plan also asks for 4 * K * roundup(M, 4) bytes in which every run
  * writes x transposed for its TMA-fed kernel (schedule only; reported as "activation_workspace_bytes"
  * by det_linear_plan_describe, not in workspace_bytes).  If that allocation fails the plan is still
  * created and runs the register-staged kernel, which computes the same bits.

@@ -124,7 +124,7 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const vo
         }
         e = launch_decode(a, cfg, &plan->map_w, &plan->map_x);
     } else if (kernel == kKernelPrefill) {
-        // 16-bit weights: the TMA-fed kernel (variant 5 .. 8 forces its rows per thread); FP32 weights, or
+        // the TMA-fed kernel (variant 5 .. 8 forces its rows per thread); without the activation workspace, or with
         // variant 15 .. 18, the register-staged kernel
         const int v = plan->variant;
         if (!plan->x_t || (v >= 15 && v <= 18)) {
@@ -136,10 +136,11 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const vo
             e = launch_transpose_x(x, plan->x_t, p.M, p.K, ldt, stream);
             if (e != cudaSuccess) return cuda_fail("kernel launch", e);
             if (plan->map_w_ptr != W || plan->map_cfg_id != cfg_id) {
-                const CUtensorMapDataType wdt = p.weight_format == DET_WEIGHT_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
-                                                                                   : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-                if (!encode_2d(&plan->map_w, wdt, 2, W, (uint64_t)plan->n_count, (uint64_t)p.K, 128u, 32u,
-                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+                const CUtensorMapDataType wdt = p.weight_format == DET_WEIGHT_FP32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                : p.weight_format == DET_WEIGHT_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                                                     : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+                if (!encode_2d(&plan->map_w, wdt, p.weight_format == DET_WEIGHT_FP32 ? 4 : 2, W, (uint64_t)plan->n_count, (uint64_t)p.K,
+                               128u, 32u, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
                     return DET_ERR_CUDA;
                 if (!encode_2d(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, plan->x_t, (uint64_t)p.K, (uint64_t)ldt, 32u,
                                (uint32_t)(16 * tr), CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
@@ -226,9 +227,9 @@ det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K, int64_
         det_linear_plan_destroy(plan);              // frees whatever was allocated before the failure
         return nullptr;
     }
-    // Activation workspace of the TMA-fed prefill kernel (16-bit weights): x transposed, 4 K roundup(M, 4) bytes.
+    // Activation workspace of the TMA-fed prefill kernel: x transposed, 4 K roundup(M, 4) bytes.
     // Without it the plan still works: it uses the register-staged kernel, which computes the same bits.
-    if (prm.kernel == kKernelPrefill && wfmt != DET_WEIGHT_FP32) {
+    if (prm.kernel == kKernelPrefill) {
         e = device_alloc(reinterpret_cast<void**>(&plan->x_t), 4ull * (uint64_t)((M + 3) / 4 * 4) * (uint64_t)K);
         if (e != cudaSuccess) { plan->x_t = nullptr; cudaGetLastError(); }
     }

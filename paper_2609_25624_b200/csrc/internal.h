@@ -53,11 +53,12 @@ cudaError_t launch_generic(const LaunchArgs& a, int bucket);
 // Second pass of split-K: y[m,n] = (((P0 + P1) + P2) + ...) (+ b[n]); rule R3.
 cudaError_t launch_combine(const LaunchArgs& a);
 
-// Register-staged prefill kernel (any weight format; a.variant 15 .. 18 forces 5 .. 8 rows per thread).
+// Register-staged prefill kernel (the fallback without an activation workspace; a.variant 15 .. 18 forces 5 .. 8 rows
+// per thread).
 cudaError_t launch_prefill(const LaunchArgs& a);
-// Prefill kernel for the 16-bit weight formats with both tiles fed by TMA (prefill_tma.cu).  It reads the
+// Prefill kernel with both tiles fed by TMA (prefill_tma.cu).  It reads the
 // activations from a workspace xT [K][ldt] (x transposed, ldt = M rounded up to a multiple of 4; launch_transpose_x
-// writes it).  Tensor maps without swizzle: map_x: xT, box [32][16 tr]; map_w: W [N][K] 16-bit, box [128][32].
+// writes it).  Tensor maps without swizzle: map_x: xT, box [32][16 tr]; map_w: W [N][K] in its format, box [128][32].
 cudaError_t launch_transpose_x(const float* x, float* xT, int64_t M, int64_t K, int64_t ldt, cudaStream_t stream);
 cudaError_t launch_prefill_tma(const LaunchArgs& a, int tr, const CUtensorMap* map_w, const CUtensorMap* map_x);
 // rows per thread (tile height = 16 x this) the prefill kernel uses for batch size M; schedule only
@@ -94,7 +95,7 @@ struct det_linear_plan {
     int device;
     int sm_count;
     float* partials;                 // device, S*M*n_count floats or nullptr
-    float* x_t;                      // device, K * roundup(M, 4) floats: x transposed (prefill bucket, 16-bit weights) or nullptr
+    float* x_t;                      // device, K * roundup(M, 4) floats: x transposed (prefill bucket) or nullptr
     int64_t n_begin, n_count, ldy;   // column shard computed by this plan (0, N, N for a whole layer)
     detlin::DeviceStatus* status;    // device
     float* x_stage;                  // device staging for det_linear_run_host

@@ -1,4 +1,5 @@
-// Prefill kernel (bucket M > 64): register-tiled FP32 GEMM on the CUDA cores (rule R1: IEEE FMA only,
+// Register-staged prefill kernel (bucket M > 64; the fallback of plans without an activation workspace, see
+// prefill_tma.cu for the kernel that normally runs): register-tiled FP32 GEMM on the CUDA cores (rule R1: IEEE FMA only,
 // never tensor cores) in the frozen prefill order (V=1, L=1, P=1): every output is one accumulation
 // chain per K segment, strictly ascending in k (the order of the paper's own kernels, supplement C on
 // rule R2); segments are summed in ascending order and the bias comes last.

@@ -1,4 +1,4 @@
-// Prefill kernel for 16-bit weights (bucket M > 64): register-tiled FP32 GEMM on the CUDA cores (rule R1:
+// Prefill kernel (bucket M > 64): register-tiled FP32 GEMM on the CUDA cores (rule R1:
 // IEEE FMA only, never tensor cores) in the frozen prefill order (V=1, L=1, P=1): every output is one
 // accumulation chain per K segment, strictly ascending in k; segments are summed in ascending order and
 // the bias comes last (rule R3).
@@ -16,7 +16,7 @@
 //     [32 k][16 TR rows] of it to shared memory.  No thread spends registers, loads, stores, address
 //     arithmetic or bounds checks on staging activations, and the multiply loop keeps few values live (the
 //     128-register budget of two blocks per SM otherwise forces the compiler to recompute addresses);
-//   * the weight tile arrives by TMA too, in its stored 16-bit format; it has to become FP32 (Eq. 2: the
+//   * the weight tile arrives by TMA too, in its stored format; it has to become FP32 (Eq. 2: the
 //     upcast is exact) and k-major, so that one 16-byte load yields two (n, n+1) operand pairs.  Each thread
 //     converts 16 weights per slab: one 16-byte shared load, eight widenings and eight stores, twice.  TMA
 //     fills out-of-range rows and columns with zeros, so there are no bounds checks;
@@ -42,10 +42,12 @@ using namespace pipe;
 constexpr int BN = 128, BK = 32;
 constexpr int kThreads = 256;
 constexpr int kXStages = 2;                          // activation stages (slab parity)
-constexpr int kRawBytes = BN * BK * 2;               // raw weight stage: [128 rows][32 k] 16-bit, 64-byte rows
+// raw weight stage: [128 rows][32 k] in the stored format (64-byte rows for 16-bit weights, 128-byte rows for FP32)
+template <int WF> struct Raw { static constexpr int kBytes = BN * BK * WeightElem<WF>::bytes; };
 constexpr int kWfBytes = BK * BN * 4;                // converted weight buffer: [32 k][128 n] FP32, columns swizzled
 
-template <int TR> struct Tile {
+template <int WF, int TR> struct Tile {
+    static constexpr int kRawBytes = Raw<WF>::kBytes;
     static constexpr int BM = 16 * TR;
     static constexpr int kXBytes = BK * BM * 4;      // [32 k][BM rows] FP32
     // stages and buffers, then barriers and the abort word; 128 bytes of slack to align the first stage
@@ -84,7 +86,8 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
                    int tiles_m, int tiles_n, long long ldy, DeviceStatus* status, unsigned long long wait_limit_ns,
                    int test_flags)
 {
-    typedef Tile<TR> T;
+    typedef Tile<WF, TR> T;
+    constexpr int kRawBytes = T::kRawBytes;
     constexpr int TB = TR - 4;                       // rows of a thread in the upper group (1 .. 4)
     extern __shared__ unsigned char smem_raw[];
     const uint32_t xring = (smem_u32(smem_raw) + 127u) & ~127u;
@@ -137,12 +140,23 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     //   the converted buffer; inside a k row the 16-byte column group g = r >> 2 is stored at g ^ 2 c, which makes
     //   the 32 lanes of a store (8 rows x 4 octets) hit 32 different banks.  The multiply loop reads whole
     //   groups at one k, so the swizzle costs it one exclusive-or per octet.
-    uint32_t cv_src[2], cv_dst[2];
+    // FP32 weights: 128 rows x 8 quads (4 weights = 16 bytes), piece p = tid + 256 j (j = 0 .. 3): row r = p >> 3, quad
+    //   c = p & 7; weight (r, k = 4 c + e) goes to k row 4 c + e with the same column swizzle g ^ 2 (k >> 3) (the two
+    //   quads of an octet then collide pairwise in a store: 16 stores per thread and slab, two-way conflicts).
+    constexpr int NP = (WF == 2) ? 4 : 2;            // 16-byte pieces per thread and slab
+    uint32_t cv_src[NP], cv_dst[NP];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        const int p = tid + 256 * j, r = p >> 2, c = p & 3;
-        cv_src[j] = (uint32_t)(r * 64 + c * 16);
-        cv_dst[j] = (uint32_t)((8 * c) * BN + ((((r >> 2) ^ (2 * c)) << 2) | (r & 3))) * 4u;
+    for (int j = 0; j < NP; ++j) {
+        const int p = tid + 256 * j;
+        if constexpr (WF == 2) {
+            const int r = p >> 3, c = p & 7;
+            cv_src[j] = (uint32_t)(r * 128 + c * 16);
+            cv_dst[j] = (uint32_t)((4 * c) * BN + ((((r >> 2) ^ (2 * (c >> 1))) << 2) | (r & 3))) * 4u;
+        } else {
+            const int r = p >> 2, c = p & 3;
+            cv_src[j] = (uint32_t)(r * 64 + c * 16);
+            cv_dst[j] = (uint32_t)((8 * c) * BN + ((((r >> 2) ^ (2 * c)) << 2) | (r & 3))) * 4u;
+        }
     }
     // Slabs alternate between two sets of buffers; the parity P of a slab is a compile-time constant of the code
     // that handles it (the slab loop is unrolled by two), so every shared-memory address of the multiply loop is a
@@ -151,17 +165,24 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         constexpr int P = decltype(par)::value;
         if (!mbar_wait(wfull0 + 8 * P, (uint32_t)(slab >> 1) & 1u, abort_flag, status, wait_limit_ns, 3)) return false;
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < NP; ++j) {
             const uint4 v = lds128u(raw0 + P * kRawBytes + cv_src[j]);
             const uint32_t a = wf0 + P * kWfBytes + cv_dst[j];
-            sts32(a, up16_lo<WF>(v.x));
-            sts32(a + 1 * BN * 4, up16_hi<WF>(v.x));
-            sts32(a + 2 * BN * 4, up16_lo<WF>(v.y));
-            sts32(a + 3 * BN * 4, up16_hi<WF>(v.y));
-            sts32(a + 4 * BN * 4, up16_lo<WF>(v.z));
-            sts32(a + 5 * BN * 4, up16_hi<WF>(v.z));
-            sts32(a + 6 * BN * 4, up16_lo<WF>(v.w));
-            sts32(a + 7 * BN * 4, up16_hi<WF>(v.w));
+            if constexpr (WF == 2) {
+                sts32(a, __uint_as_float(v.x));
+                sts32(a + 1 * BN * 4, __uint_as_float(v.y));
+                sts32(a + 2 * BN * 4, __uint_as_float(v.z));
+                sts32(a + 3 * BN * 4, __uint_as_float(v.w));
+            } else {
+                sts32(a, up16_lo<WF>(v.x));
+                sts32(a + 1 * BN * 4, up16_hi<WF>(v.x));
+                sts32(a + 2 * BN * 4, up16_lo<WF>(v.y));
+                sts32(a + 3 * BN * 4, up16_hi<WF>(v.y));
+                sts32(a + 4 * BN * 4, up16_lo<WF>(v.z));
+                sts32(a + 5 * BN * 4, up16_hi<WF>(v.z));
+                sts32(a + 6 * BN * 4, up16_lo<WF>(v.w));
+                sts32(a + 7 * BN * 4, up16_hi<WF>(v.w));
+            }
         }
         return true;
     };
@@ -181,10 +202,12 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
     for (int c = 0; c < 4; ++c) w_oct[c] = wf0 + (uint32_t)(8 * c * BN) * 4u + (uint32_t)((tx ^ (2 * c)) << 4);
 
-    // one octet of k: k = 8 c + e inside the slab
-    auto octet = [&](uint32_t xlo, uint32_t xhi, uint32_t wc) {
+    // one octet of k: k = 8 c + e inside the slab (ne = 8; ne = 4 for the last four k of an FP32-weight layer whose K is
+    // a multiple of 4 only)
+    auto octet = [&](uint32_t xlo, uint32_t xhi, uint32_t wc, auto ne_c) {
+        constexpr int NE = decltype(ne_c)::value;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
+        for (int e = 0; e < NE; ++e) {
             float xv[TR];
             lds_floats<4>(xlo + (uint32_t)(e * T::BM) * 4u, xv);
             lds_floats<TB>(xhi + (uint32_t)(e * T::BM) * 4u, xv + 4);
@@ -206,18 +229,27 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         bool ok = true;
         if (slab + 1 < n_slabs) ok = convert(slab + 1, std::integral_constant<int, P ^ 1>());
         if (ok) ok = mbar_wait(xfull0 + 8 * P, (uint32_t)(slab >> 1) & 1u, abort_flag, status, wait_limit_ns, 4);
-        // k beyond the end of the segment is skipped, not zero-filled; segments end on multiples of 8
-        const int n_oct = ok ? (min(BK, k_hi - (k_lo + slab * BK)) >> 3) : 0;
+        // k beyond the end of the segment is skipped, not zero-filled; segments end on multiples of 8 (16-bit weights)
+        // or 4 (FP32 weights)
+        const int n_k = ok ? min(BK, k_hi - (k_lo + slab * BK)) : 0;
+        const int n_oct = n_k >> 3;
+        using Eight = std::integral_constant<int, 8>;
+        using Four = std::integral_constant<int, 4>;
         if (n_oct == 4) {
 #pragma unroll
             for (int c = 0; c < 4; ++c)
                 octet(x_lo + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u, x_hi + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u,
-                      w_oct[c] + P * kWfBytes);
+                      w_oct[c] + P * kWfBytes, Eight());
         } else {
 #pragma unroll 1
             for (int c = 0; c < n_oct; ++c)
                 octet(x_lo + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u, x_hi + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u,
-                      wf0 + P * kWfBytes + (uint32_t)(8 * c * BN) * 4u + (uint32_t)((tx ^ (2 * c)) << 4));
+                      wf0 + P * kWfBytes + (uint32_t)(8 * c * BN) * 4u + (uint32_t)((tx ^ (2 * c)) << 4), Eight());
+            if (WF == 2 && (n_k & 4)) {
+                const int c = n_oct;
+                octet(x_lo + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u, x_hi + P * T::kXBytes + (uint32_t)(8 * c * T::BM) * 4u,
+                      wf0 + P * kWfBytes + (uint32_t)(8 * c * BN) * 4u + (uint32_t)((tx ^ (2 * c)) << 4), Four());
+            }
         }
         // the barrier carries the vote
         if (!__syncthreads_and(ok)) return false;
@@ -287,7 +319,7 @@ __global__ void __launch_bounds__(256) transpose_x_kernel(const float* __restric
 template <int WF, int TR>
 cudaError_t launch_t(const LaunchArgs& a, const CUtensorMap* map_w, const CUtensorMap* map_x)
 {
-    typedef Tile<TR> T;
+    typedef Tile<WF, TR> T;
     static bool configured[kMaxDevices];             // function attributes belong to a device
     int dev = 0;
     cudaError_t de = cudaGetDevice(&dev);
@@ -345,6 +377,7 @@ cudaError_t launch_prefill_tma(const LaunchArgs& a, int tr, const CUtensorMap* m
     switch (a.wfmt) {
     case DET_WEIGHT_BF16: return launch_f<0>(a, tr, map_w, map_x);
     case DET_WEIGHT_FP16: return launch_f<1>(a, tr, map_w, map_x);
+    case DET_WEIGHT_FP32: return launch_f<2>(a, tr, map_w, map_x);
     default: return cudaErrorInvalidValue;
     }
 }
