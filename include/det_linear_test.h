@@ -50,7 +50,9 @@ DET_API void det_test_attention_set_split(int blocks_per_row);
  * into the bound.  The
  * kernel then records the timeout in the plan's status word, drains and returns (no trap, no endless
  * loop; the other blocks finish normally), and det_linear_plan_check reports DET_ERR_DEVICE_TIMEOUT.
- * The output of such a run is undefined.  Reset with (2000000000, 0).
+ * The output of such a run is undefined.  Bit 1 (value 2) makes a prefill plan with several K segments fold them
+ * with the second (combine) launch instead of inside the kernel: same bits, another schedule.
+ * Reset with (2000000000, 0).
  */
 DET_API det_status_t det_test_plan_set_wait(det_linear_plan_t* plan, uint64_t wait_limit_ns, int flags);
 

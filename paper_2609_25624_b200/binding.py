@@ -367,9 +367,10 @@ def det_test_fail_next_alloc(nth: int = 1) -> None:
     lib().det_test_fail_next_alloc(int(nth))
 
 
-def det_test_plan_set_wait(plan: Plan, wait_limit_ns: int, withhold_first_copy: bool = False) -> None:
-    """Bound of one device-side wait for this plan's kernels; optionally stall one wait on purpose."""
-    flags = 1 if withhold_first_copy else 0
+def det_test_plan_set_wait(plan: Plan, wait_limit_ns: int, withhold_first_copy: bool = False, two_pass_combine: bool = False) -> None:
+    """Bound of one device-side wait for this plan's kernels; optionally stall one wait on purpose; optionally make a
+    prefill plan fold its K segments with the second launch instead of inside the kernel (same bits)."""
+    flags = (1 if withhold_first_copy else 0) | (2 if two_pass_combine else 0)
     _check(lib().det_test_plan_set_wait(plan.handle, int(wait_limit_ns), flags))
 
 

@@ -82,6 +82,10 @@ static det_status_t run_device(det_linear_plan_t* plan, const float* x, const vo
     a.x = x; a.W = W; a.b = b; a.y = y;
     a.wfmt = p.weight_format;
     a.partials = plan->partials;
+    // Prefill with 2 .. 4 segments: the block that completes a tile folds it (measured 0.5 - 3 % faster than the second
+    // launch); with more segments the fold of a tile by one block is a longer serial tail than the combine launch
+    // (1 - 5 % slower), so that keeps the second pass.  Test flag 2 forces the second pass.  Same bits either way.
+    a.tile_counters = ((plan->test_flags & 2) || p.S > 4) ? nullptr : plan->tile_counters;
     a.M = p.M; a.N = plan->n_count; a.K = p.K;            // the kernels see the shard; the order is the layer's
     a.ldy = plan->ldy;
     a.seg_len = p.seg_len; a.S = p.S;
@@ -218,7 +222,16 @@ det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K, int64_
     g_last_status = DET_OK;
     e = device_alloc(reinterpret_cast<void**>(&plan->status), sizeof(DeviceStatus));
     if (e == cudaSuccess) e = cudaMemset(plan->status, 0, sizeof(DeviceStatus));
-    if (e == cudaSuccess && prm.workspace_bytes) e = device_alloc(reinterpret_cast<void**>(&plan->partials), prm.workspace_bytes);
+    // the partials are followed by one counter per output tile of the prefill kernel (at most ceil(M/80) ceil(N/128))
+    const uint64_t counters_at = (prm.workspace_bytes + 255) / 256 * 256;
+    const uint64_t n_counters = (uint64_t)((M + 79) / 80) * (uint64_t)((n_count + 127) / 128);
+    if (e == cudaSuccess && prm.workspace_bytes) {
+        e = device_alloc(reinterpret_cast<void**>(&plan->partials), counters_at + 4 * n_counters);
+        if (e == cudaSuccess) {
+            plan->tile_counters = reinterpret_cast<unsigned*>(reinterpret_cast<char*>(plan->partials) + counters_at);
+            e = cudaMemset(plan->tile_counters, 0, 4 * n_counters);
+        }
+    }
     if (e != cudaSuccess) {
         g_last_status = DET_ERR_ALLOC;
         set_error("plan: device allocation (status word, %llu bytes of split-K workspace) failed: %s",
@@ -543,7 +556,7 @@ void det_test_fail_next_alloc(int nth)
 
 det_status_t det_test_plan_set_wait(det_linear_plan_t* plan, uint64_t wait_limit_ns, int flags)
 {
-    if (!plan || wait_limit_ns == 0 || flags < 0 || flags > 1) { set_error("set_wait: bad argument"); return DET_ERR_INVALID_ARG; }
+    if (!plan || wait_limit_ns == 0 || flags < 0 || flags > 3) { set_error("set_wait: bad argument"); return DET_ERR_INVALID_ARG; }
     plan->wait_limit_ns = wait_limit_ns;
     plan->test_flags = flags;
     return DET_OK;

@@ -37,6 +37,7 @@ struct LaunchArgs {
     float* y;             // final output [M,N], row pitch ldy
     int64_t ldy;          // floats between consecutive rows of y (N unless the plan is a column shard)
     float* partials;      // [S,M,N] when S > 1, else nullptr
+    unsigned* tile_counters;   // prefill with S > 1: one zeroed counter per output tile (the TMA-fed kernel folds in place), or nullptr
     int64_t M, N, K;
     int64_t seg_len;
     int S;
@@ -95,6 +96,7 @@ struct det_linear_plan {
     int device;
     int sm_count;
     float* partials;                 // device, S*M*n_count floats or nullptr
+    unsigned* tile_counters;         // device, inside the partials allocation (prefill, S > 1) or nullptr
     float* x_t;                      // device, K * roundup(M, 4) floats: x transposed (prefill bucket) or nullptr
     int64_t n_begin, n_count, ldy;   // column shard computed by this plan (0, N, N for a whole layer)
     detlin::DeviceStatus* status;    // device

@@ -84,8 +84,9 @@ __global__ void __launch_bounds__(kThreads, 2)
 prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                    const float* __restrict__ bias, float* __restrict__ out, int M, int N, int K, int seg_len, int direct,
                    int tiles_m, int tiles_n, long long ldy, DeviceStatus* status, unsigned long long wait_limit_ns,
-                   int test_flags)
+                   int test_flags, float* __restrict__ y, unsigned* __restrict__ tile_counters, int S)
 {
+    __shared__ int fold_here;                        // split-K: this block wrote the last partial of its tile
     typedef Tile<WF, TR> T;
     constexpr int kRawBytes = T::kRawBytes;
     constexpr int TB = TR - 4;                       // rows of a thread in the upper group (1 .. 4)
@@ -293,6 +294,57 @@ prefill_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             }
         }
     }
+    if (direct || tile_counters == nullptr) return;
+
+    // ---- split-K fold without a second launch (rule R3): the block that completes a tile's count of S partials adds
+    // them in ascending segment order, then the bias, and stores.  Which block that is depends on timing; what it
+    // computes does not.  Nobody waits for anybody.  The counter returns to zero for the next run. ----
+    __threadfence();                                 // this block's partials are visible before its count
+    __syncthreads();
+    if (tid == 0) {
+        unsigned* cnt = tile_counters + ((long long)tn * tiles_m + tm);
+        const unsigned before = atomicAdd(cnt, 1u);
+        fold_here = (before == (unsigned)(S - 1));
+        if (fold_here) *cnt = 0u;
+    }
+    __syncthreads();
+    if (!fold_here) return;
+    __threadfence();                                 // the other blocks' partials, counted before ours, are visible
+    const bool y_vec = (ldy % 4 == 0) && (N % 4 == 0);
+#pragma unroll 1
+    for (int i = 0; i < TR; ++i) {
+        const int m = m0 + (i < 4 ? 4 * ty + i : 64 + TB * ty + (i - 4));
+        if (m >= M) continue;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int n = n0 + 64 * h + 4 * tx;
+            if (n >= N) continue;
+            const float* p0 = out + (long long)m * N + n;
+            const long long seg_stride = (long long)M * N;
+            float v[4];
+            if (y_vec && n + 3 < N) {
+                float4 t = __ldcg(reinterpret_cast<const float4*>(p0));
+                for (int s2 = 1; s2 < S; ++s2) {
+                    const float4 u4 = __ldcg(reinterpret_cast<const float4*>(p0 + s2 * seg_stride));
+                    t.x = __fadd_rn(t.x, u4.x); t.y = __fadd_rn(t.y, u4.y); t.z = __fadd_rn(t.z, u4.z); t.w = __fadd_rn(t.w, u4.w);
+                }
+                v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+                if (bias) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) v[e] = __fadd_rn(v[e], bias[n + e]);
+                }
+                *reinterpret_cast<float4*>(y + (long long)m * ldy + n) = make_float4(v[0], v[1], v[2], v[3]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (n + e >= N) continue;
+                    float t = __ldcg(p0 + e);
+                    for (int s2 = 1; s2 < S; ++s2) t = __fadd_rn(t, __ldcg(p0 + e + s2 * seg_stride));
+                    y[(long long)m * ldy + n + e] = bias ? __fadd_rn(t, bias[n + e]) : t;
+                }
+            }
+        }
+    }
 }
 
 // First pass: xT[k][m] = x[m][k] for m < M, 0 for M <= m < ldt (ldt = M rounded up to a multiple of 4, the row pitch
@@ -336,10 +388,10 @@ cudaError_t launch_t(const LaunchArgs& a, const CUtensorMap* map_w, const CUtens
     const int direct = (a.S == 1);
     prefill_tma_kernel<WF, TR><<<(unsigned)units, kThreads, T::kSmemBytes, a.stream>>>(
         *map_x, *map_w, a.b, direct ? a.y : a.partials, (int)a.M, (int)a.N, (int)a.K, (int)a.seg_len, direct, tiles_m, tiles_n,
-        (long long)a.ldy, a.status, a.wait_limit_ns, a.test_flags);
+        (long long)a.ldy, a.status, a.wait_limit_ns, a.test_flags, a.y, a.tile_counters, a.S);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    if (!direct) return launch_combine(a);
+    if (!direct && !a.tile_counters) return launch_combine(a);
     return cudaSuccess;
 }
 

@@ -12,7 +12,7 @@ def to_dev(t):
     return None if t is None else t.cuda()
 
 
-def run_gpu(x, W, b, kernel=None, variant=0, max_blocks=0, stream=None, y_fill=float("nan")):
+def run_gpu(x, W, b, kernel=None, variant=0, max_blocks=0, stream=None, y_fill=float("nan"), two_pass_combine=False):
     """x [M,K] f32, W [N,K] bf16 / fp16 / fp32 (the plan's weight format follows the dtype), b [N] f32 or
     None (CPU or CUDA tensors) -> y as numpy float32 [M,N].
     The output buffer is pre-filled with NaN so that an element the kernel never wrote is caught."""
@@ -28,6 +28,8 @@ def run_gpu(x, W, b, kernel=None, variant=0, max_blocks=0, stream=None, y_fill=f
             B.det_test_plan_set_variant(plan, variant)
         if max_blocks:
             B.det_test_plan_set_max_blocks(plan, max_blocks)
+        if two_pass_combine:
+            B.det_test_plan_set_wait(plan, 2_000_000_000, two_pass_combine=True)
         B.det_linear_run(plan, xd, Wd, bd, y, stream=stream)
         B.det_linear_plan_check(plan, stream=stream)
         torch.cuda.synchronize()

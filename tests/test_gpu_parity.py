@@ -198,6 +198,17 @@ def test_prefill_tile_heights_bit_exact(M, N, K):
     # 5 .. 8: the TMA-fed kernel with that many rows per thread; 15 .. 18: the register-staged kernel
     for variant in (0, 5, 6, 7, 8, 15, 16, 17, 18):
         assert_bits_equal(run_gpu(x, W, b, kernel=KERNEL_PREFILL, variant=variant), want, f"rows per thread {variant}")
+    # K segments folded by the second launch instead of by the block that completes a tile
+    assert_bits_equal(run_gpu(x, W, b, kernel=KERNEL_PREFILL, two_pass_combine=True), want, "two-pass combine")
+    # the in-kernel fold leaves its tile counters at zero: a second run of the same plan gives the same bits
+    plan = B.det_linear_plan(M, N, K)
+    xd, Wd, bd = x.cuda(), W.cuda(), b.cuda()
+    for rep in range(3):
+        y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        B.det_linear_run(plan, xd, Wd, bd, y)
+        torch.cuda.synchronize()
+        assert_bits_equal(y.cpu().numpy(), want, f"repeat {rep}")
+    plan.close()
 
 
 def test_prefill_tile_choice():
