@@ -189,7 +189,9 @@ DET_API det_status_t det_linear_plan_tune(det_linear_plan_t* plan, const float* 
  * Synchronise `stream` and report whether any kernel launched through this plan gave up a bounded
  * device-side wait (every wait on a TMA completion barrier is limited; on expiry the kernel
  * records the fact and returns instead of spinning).  DET_OK, DET_ERR_DEVICE_TIMEOUT or
- * DET_ERR_CUDA.  The record is cleared by the call.
+ * DET_ERR_CUDA.  The record is cleared by the call.  After a kernel gave up, the outputs of that run are
+ * undefined and the plan must pass through this call (which also resets the plan's split-K bookkeeping)
+ * before it is used again.
  */
 DET_API det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream);
 

@@ -229,6 +229,7 @@ det_linear_plan_t* det_linear_plan_shard(int64_t M, int64_t N, int64_t K, int64_
         e = device_alloc(reinterpret_cast<void**>(&plan->partials), counters_at + 4 * n_counters);
         if (e == cudaSuccess) {
             plan->tile_counters = reinterpret_cast<unsigned*>(reinterpret_cast<char*>(plan->partials) + counters_at);
+            plan->n_tile_counters = n_counters;
             e = cudaMemset(plan->tile_counters, 0, 4 * n_counters);
         }
     }
@@ -433,6 +434,12 @@ det_status_t det_linear_plan_check(det_linear_plan_t* plan, void* stream)
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail("check", e);
     if (h.timeout_flag) {
+        // a block that gave up did not count itself in: bring the tile counters of the in-kernel fold back to zero
+        if (plan->tile_counters) {
+            e = cudaMemsetAsync(plan->tile_counters, 0, 4 * plan->n_tile_counters, st);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+            if (e != cudaSuccess) return cuda_fail("check", e);
+        }
         set_error("check: a kernel gave up a bounded wait (site %u)", h.where);
         return DET_ERR_DEVICE_TIMEOUT;
     }

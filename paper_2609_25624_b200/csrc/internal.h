@@ -97,6 +97,7 @@ struct det_linear_plan {
     int sm_count;
     float* partials;                 // device, S*M*n_count floats or nullptr
     unsigned* tile_counters;         // device, inside the partials allocation (prefill, S > 1) or nullptr
+    uint64_t n_tile_counters;
     float* x_t;                      // device, K * roundup(M, 4) floats: x transposed (prefill bucket) or nullptr
     int64_t n_begin, n_count, ldy;   // column shard computed by this plan (0, N, N for a whole layer)
     detlin::DeviceStatus* status;    // device
