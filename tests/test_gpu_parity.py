@@ -268,3 +268,18 @@ def test_prefill_very_tall_batches(M, N, K):
     plan.close()
     assert_bits_equal(run_gpu(x, W, b), want, "automatic")
     assert_bits_equal(run_gpu(x, W, b, variant=18), want, "register-staged")
+
+
+@pytest.mark.parametrize("M,N,K", [(130, 40, 8), (70, 16, 24), (200, 8, 40), (66, 300, 32), (129, 129, 72)])
+def test_prefill_very_short_k(M, N, K):
+    """One or two slabs of K, shorter than a slab, not a multiple of it: the TMA-fed kernel against the oracle,
+    every element, for BF16 and for FP32 weights (K a multiple of 8 serves both)."""
+    x, W, b = inputs.make_case(M, N, K)
+    want = oracle_y(x, W, b)
+    assert_bits_equal(run_gpu(x, W, b, kernel=KERNEL_PREFILL), want, "bf16")
+    W32 = W.float()
+    assert_bits_equal(run_gpu(x, W32, b, kernel=KERNEL_PREFILL), oracle_y(x, W32, b), "fp32 weights")
+    if K % 8 == 0 and K >= 12:
+        W32s = W32[:, : K - 4].contiguous()             # K a multiple of 4 only: the four-element tail
+        xs = x[:, : K - 4].contiguous()
+        assert_bits_equal(run_gpu(xs, W32s, b, kernel=KERNEL_PREFILL), oracle_y(xs, W32s, b), "fp32 weights, K % 8 == 4")
