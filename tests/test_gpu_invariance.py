@@ -14,7 +14,10 @@ from tests.gpu_util import assert_bits_equal, oracle_y, run_gpu
 
 pytestmark = pytest.mark.gpu
 
-CASES = [(1, 1024, 512), (8, 4096, 4096), (32, 1000, 2048), (130, 520, 2304)]
+# decode (M <= 64) and prefill; the prefill cases cover the combine launch (S = 9) and the in-kernel fold, where the
+# block that folds a tile is whichever finishes last (S = 4, 3, 2)
+CASES = [(1, 1024, 512), (8, 4096, 4096), (32, 1000, 2048), (130, 520, 2304), (200, 1024, 1024), (300, 1152, 768),
+         (512, 640, 512)]
 
 
 def digest(t):
