@@ -36,7 +36,7 @@ DET_API det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int vari
 DET_API void det_test_fail_next_alloc(int nth);
 
 /*
- * det_attention_decode spreads the keys of one (batch, KV head) row over a cluster of 1, 2, 4 or 8 thread
+ * det_attention_decode spreads the keys of one (batch, KV head) row over a cluster of 1, 2, 4, 8 or 16 thread
  * blocks, chosen from the shape and the SM count (schedule only: every choice gives the same bits).  This
  * forces the choice for the calls that follow (capped by the number of 256-key segments of the row);
  * 0 = automatic again.  Process-wide: tests only.

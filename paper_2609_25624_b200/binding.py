@@ -358,7 +358,7 @@ def det_test_plan_set_variant(plan: Plan, variant: int) -> None:
 
 
 def det_test_attention_set_split(blocks_per_row: int) -> None:
-    """Force the cluster size of det_attention_decode (1, 2, 4, 8; 0 = automatic).  Same bits for every value."""
+    """Force the cluster size of det_attention_decode (1, 2, 4, 8, 16; 0 = automatic).  Same bits for every value."""
     lib().det_test_attention_set_split(blocks_per_row)
 
 

@@ -14,7 +14,7 @@
 //   5. for every d: keys in segments of 256; inside a segment a = fma.rn(e_j, v_j[d], a) from +0 with j
 //      ascending; segment sums added left to right in ascending order; o[d] = sum / l (one div.rn).
 //
-// Schedule (numerically inert): a cluster of C thread blocks (C = 1, 2, 4 or 8) per (batch, KV head) serves
+// Schedule (numerically inert): a cluster of C thread blocks (C = 1, 2, 4, 8 or 16) per (batch, KV head) serves
 // the G = Hq / Hkv query heads that share the head's keys and values, so K and V cross the memory bus once
 // per group.  Block r of the cluster owns the keys [r Tc, (r + 1) Tc), Tc a whole number of 256-key
 // segments; everything that crosses the blocks goes through distributed shared memory behind hardware
@@ -39,6 +39,7 @@ constexpr int kAttnThreads = 256;
 constexpr int kAttnWarps = kAttnThreads / 32;
 constexpr int kKeysPerPass = 8;          // keys a warp scores together
 constexpr int kSegKeys = 256;            // P.V segment length (part of the order)
+constexpr int kMaxCluster = 16;          // blocks per row at most (8 is the portable cluster size, 16 needs the opt-in below)
 
 // The attention's exponential for x <= 0: range reduction by ln 2 in two pieces, degree-7 Taylor polynomial
 // by Horner's rule with fused multiply-adds, scaling by 2^n (through 2^(n+64) and 2^-64 below the normal
@@ -360,6 +361,7 @@ cudaError_t launch_attention_t(const float* q, const float* k, const float* v, f
     auto kern = attention_decode_kernel<G, DC>;
     if (!configured[dev]) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);   // clusters of 16
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -403,10 +405,14 @@ int attention_split(int B, int Hkv, int G, int T, int D, int sm_count)
 {
     const int n_seg = (T + kSegKeys - 1) / kSegKeys;
     int c_max = 1;
-    while (c_max < 8 && 2 * c_max <= n_seg) c_max *= 2;
+    while (c_max < kMaxCluster && 2 * c_max <= n_seg) c_max *= 2;
     if (g_attention_force_split) return g_attention_force_split <= c_max ? g_attention_force_split : c_max;
+    // clusters of 16 (not portable, one GPC each) only pay for very few, very long rows (measured: 8 rows of 16384 keys
+    // or more; 16 rows, or 4096 keys, are faster in clusters of 8)
+    const bool few_long_rows = (long long)B * Hkv * 16 <= sm_count && n_seg >= 64;
+    const int c_auto = (c_max > 8 && !few_long_rows) ? 8 : c_max;
     int c = 1;
-    while (c < c_max && (long long)B * Hkv * (2 * c) <= 2ll * sm_count) c *= 2;
+    while (c < c_auto && (long long)B * Hkv * (2 * c) <= 2ll * sm_count) c *= 2;
     while (c < c_max && block_smem_bytes(G, keys_per_block(T, c), D) > 110u * 1024u) c *= 2;
     return c;
 }
@@ -416,11 +422,11 @@ size_t attention_smem_bytes(int G, int T, int D)
 {
     const int n_seg = (T + kSegKeys - 1) / kSegKeys;
     int c_max = 1;
-    while (c_max < 8 && 2 * c_max <= n_seg) c_max *= 2;
+    while (c_max < kMaxCluster && 2 * c_max <= n_seg) c_max *= 2;
     return block_smem_bytes(G, keys_per_block(T, c_max), D);
 }
 
-void attention_test_force_split(int c) { g_attention_force_split = (c == 1 || c == 2 || c == 4 || c == 8) ? c : 0; }
+void attention_test_force_split(int c) { g_attention_force_split = (c == 1 || c == 2 || c == 4 || c == 8 || c == 16) ? c : 0; }
 
 cudaError_t launch_attention_decode(const float* q, const float* k, const float* v, float scale, int B, int Hq, int Hkv, int T, int D,
                                     float* o, cudaStream_t stream)
@@ -431,7 +437,7 @@ cudaError_t launch_attention_decode(const float* q, const float* k, const float*
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         sms = 148;
     int C = attention_split(B, Hkv, G, T, D, sms);
-    while (C < 8 && block_smem_bytes(G, keys_per_block(T, C), D) > 227u * 1024u) C *= 2;   // must fit at all
+    while (C < kMaxCluster && block_smem_bytes(G, keys_per_block(T, C), D) > 227u * 1024u) C *= 2;   // must fit at all
     const int Tc = keys_per_block(T, C);
     const size_t smem = block_smem_bytes(G, Tc, D);
     if (smem > 227u * 1024u) return cudaErrorInvalidValue;

@@ -68,7 +68,7 @@ int prefill_rows_per_thread(int64_t M);
 cudaError_t launch_rmsnorm(const float* x, const float* g, float eps, int64_t M, int64_t H, float* y, cudaStream_t stream);
 // Fixed-order decode attention (attention.cu); attention_smem_bytes = dynamic shared memory it needs.
 size_t attention_smem_bytes(int G, int T, int D);
-// test hook: force the number of thread blocks that share one (batch, KV head) row (1, 2, 4, 8; 0 = automatic)
+// test hook: force the number of thread blocks that share one (batch, KV head) row (1, 2, 4, 8, 16; 0 = automatic)
 void attention_test_force_split(int c);
 cudaError_t launch_attention_decode(const float* q, const float* k, const float* v, float scale, int B, int Hq, int Hkv, int T,
                                     int D, float* o, cudaStream_t stream);

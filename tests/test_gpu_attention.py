@@ -46,15 +46,15 @@ def test_attention_bit_exact(B_, Hq, Hkv, T, D):
 
 
 @pytest.mark.parametrize("B_,Hq,Hkv,T,D", [(2, 8, 2, 1000, 128), (1, 32, 8, 2049, 128), (3, 4, 4, 513, 96), (1, 8, 1, 4096, 128),
-                                           (2, 2, 1, 260, 256), (1, 8, 2, 255, 128)])
+                                           (2, 2, 1, 260, 256), (1, 8, 2, 255, 128), (1, 4, 1, 16500, 64)])
 def test_attention_same_bits_for_every_cluster_size(B_, Hq, Hkv, T, D):
-    """The keys of a row are spread over 1, 2, 4 or 8 thread blocks (row maxima, denominators and segment sums meet
+    """The keys of a row are spread over 1, 2, 4, 8 or 16 thread blocks (row maxima, denominators and segment sums meet
     through distributed shared memory): schedule only, every cluster size reproduces the oracle's bits."""
     q, k, v = make_qkv(B_, Hq, Hkv, T, D, seed=T + D)
     scale = float(np.float32(1.0 / math.sqrt(D)))
     want = oracle.attention_decode(q.numpy(), k.numpy(), v.numpy(), scale)
     try:
-        for c in (1, 2, 4, 8, 0):
+        for c in (1, 2, 4, 8, 16, 0):
             B.det_test_attention_set_split(c)
             assert_bits_equal(run_gpu_attention(q, k, v, scale), want, f"cluster of {c}")
     finally:
@@ -104,7 +104,7 @@ def test_attention_argument_checks():
     with pytest.raises(B.DetLinearError) as ei:
         B.det_attention_decode(q.cuda(), k.cuda(), v.cuda(), 1.0, o)
     assert ei.value.status == 2
-    q, k, v = make_qkv(1, 4, 1, 100000, 128, seed=1)          # scores do not fit in shared memory, however the row is split
+    q, k, v = make_qkv(1, 4, 1, 200000, 128, seed=1)          # scores do not fit in shared memory, however the row is split
     o = torch.empty(1, 4, 128, device="cuda")
     with pytest.raises(B.DetLinearError) as ei:
         B.det_attention_decode(q.cuda(), k.cuda(), v.cuda(), 1.0, o)
