@@ -42,6 +42,11 @@ DET_API void det_test_fail_next_alloc(int nth);
  * 0 = automatic again.  Process-wide: tests only.
  */
 DET_API void det_test_attention_set_split(int blocks_per_row);
+/* The cluster size det_attention_decode would use for this shape on a device with sm_count SMs, and the dynamic
+ * shared memory of one block for it (*smem_bytes_out, may be NULL; above 232448 the call would be refused).
+ * Host arithmetic only: touches no device.  0 on bad arguments. */
+DET_API int det_test_attention_schedule(int64_t B, int64_t Hq, int64_t Hkv, int64_t T, int64_t D, int sm_count,
+                                        uint64_t* smem_bytes_out);
 
 /*
  * Bound of one device-side wait for the kernels launched through this plan (default 2 s), and flags:

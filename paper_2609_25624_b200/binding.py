@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.det_last_error.restype = ctypes.c_char_p
         L.det_order_version.restype = i32
         L.det_last_status.restype = i32
+        L.det_test_attention_schedule.argtypes = [i64, i64, i64, i64, i64, i32, ctypes.POINTER(ctypes.c_uint64)]
+        L.det_test_attention_schedule.restype = i32
         L.det_test_attention_set_split.argtypes = [i32]
         L.det_test_attention_set_split.restype = None
         L.det_test_fail_next_alloc.argtypes = [i32]
@@ -355,6 +357,13 @@ def det_test_plan_set_max_blocks(plan: Plan, max_blocks: int) -> None:
 
 def det_test_plan_set_variant(plan: Plan, variant: int) -> None:
     _check(lib().det_test_plan_set_variant(plan.handle, variant))
+
+
+def det_test_attention_schedule(B_: int, Hq: int, Hkv: int, T: int, D: int, sm_count: int = 148):
+    """(cluster size, shared-memory bytes per block) det_attention_decode would use; host arithmetic only."""
+    smem = ctypes.c_uint64(0)
+    c = lib().det_test_attention_schedule(B_, Hq, Hkv, T, D, sm_count, ctypes.byref(smem))
+    return c, smem.value
 
 
 def det_test_attention_set_split(blocks_per_row: int) -> None:

@@ -426,6 +426,8 @@ size_t attention_smem_bytes(int G, int T, int D)
     return block_smem_bytes(G, keys_per_block(T, c_max), D);
 }
 
+size_t attention_block_smem_bytes(int G, int T, int D, int C) { return block_smem_bytes(G, keys_per_block(T, C), D); }
+
 void attention_test_force_split(int c) { g_attention_force_split = (c == 1 || c == 2 || c == 4 || c == 8 || c == 16) ? c : 0; }
 
 cudaError_t launch_attention_decode(const float* q, const float* k, const float* v, float scale, int B, int Hq, int Hkv, int T, int D,

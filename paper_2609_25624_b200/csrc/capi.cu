@@ -556,6 +556,16 @@ det_status_t det_test_plan_set_variant(det_linear_plan_t* plan, int variant)
 
 void det_test_attention_set_split(int blocks_per_row) { attention_test_force_split(blocks_per_row); }
 
+int det_test_attention_schedule(int64_t B, int64_t Hq, int64_t Hkv, int64_t T, int64_t D, int sm_count, uint64_t* smem_bytes_out)
+{
+    if (B < 1 || Hq < 1 || Hkv < 1 || T < 1 || D < 1 || Hq % Hkv != 0 || sm_count < 1) return 0;
+    const int G = (int)(Hq / Hkv);
+    int C = attention_split((int)B, (int)Hkv, G, (int)T, (int)D, sm_count);
+    while (C < 16 && attention_block_smem_bytes(G, (int)T, (int)D, C) > 227u * 1024u) C *= 2;
+    if (smem_bytes_out) *smem_bytes_out = attention_block_smem_bytes(G, (int)T, (int)D, C);
+    return C;
+}
+
 void det_test_fail_next_alloc(int nth)
 {
     g_fail_alloc_countdown = nth > 0 ? nth : 0;

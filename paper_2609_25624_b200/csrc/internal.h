@@ -70,6 +70,10 @@ cudaError_t launch_rmsnorm(const float* x, const float* g, float eps, int64_t M,
 size_t attention_smem_bytes(int G, int T, int D);
 // test hook: force the number of thread blocks that share one (batch, KV head) row (1, 2, 4, 8, 16; 0 = automatic)
 void attention_test_force_split(int c);
+// the cluster size the launcher would use on a device with sm_count SMs (pure function of its arguments and of
+// the forced split), and the dynamic shared memory of one block for it
+int attention_split(int B, int Hkv, int G, int T, int D, int sm_count);
+size_t attention_block_smem_bytes(int G, int T, int D, int C);
 cudaError_t launch_attention_decode(const float* q, const float* k, const float* v, float scale, int B, int Hq, int Hkv, int T,
                                     int D, float* o, cudaStream_t stream);
 // Read `bytes` at buf through L2 (evicts what was there without leaving dirty lines); sink: 4 bytes of device memory.

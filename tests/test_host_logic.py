@@ -56,6 +56,31 @@ def test_plan_params_rule_and_oracle_agree(built_lib):
         assert B.det_linear_plan_params(M, 1024, 512).as_dict() == ref
 
 
+def test_attention_cluster_rule(built_lib):
+    """The number of thread blocks that share one (batch, KV head) row of the decode attention is host arithmetic:
+    one resident wave of two blocks per SM, never more blocks than 256-key segments, 16 only for few very long
+    rows, more blocks when the scores of a block would not fit two to an SM."""
+    B = built_lib
+    sched = B.det_test_attention_schedule
+    assert sched(32, 32, 8, 2048, 128)[0] == 1            # 256 rows fill 148 SMs twice over
+    assert sched(16, 32, 8, 2048, 128)[0] == 2
+    assert sched(8, 32, 8, 4096, 128)[0] == 4
+    assert sched(4, 32, 8, 4096, 128)[0] == 8
+    assert sched(1, 32, 8, 4096, 128)[0] == 8             # 16 segments, but 16-block clusters only from 64 segments on
+    assert sched(1, 32, 8, 65536, 128)[0] == 16
+    assert sched(2, 32, 8, 32768, 128)[0] == 8            # 16 rows: clusters of 8
+    assert sched(1, 32, 8, 300, 128)[0] == 2              # two segments: at most two blocks
+    assert sched(1, 8, 8, 1, 128)[0] == 1
+    c, smem = sched(32, 32, 8, 8192, 128)                 # one block per row would need 164 KB: split in two
+    assert c == 2 and smem <= 110 * 1024
+    c, smem = sched(1, 4, 1, 131072, 128)
+    assert c == 16 and smem <= 227 * 1024
+    c, smem = sched(1, 4, 1, 200000, 128)                 # does not fit however it is split: the call is refused
+    assert c == 16 and smem > 227 * 1024
+    assert sched(8, 32, 8, 4096, 128, 74)[0] == 2         # half the SMs: half the blocks
+    assert sched(0, 32, 8, 4096, 128)[0] == 0
+
+
 def test_bad_shapes_are_rejected_with_a_message(built_lib):
     B = built_lib
     for shp in [(0, 1, 1), (1, 0, 1), (1, 1, 0), (-3, 4, 8), (1, 1 << 31, 8), (1 << 21, 1 << 21, 8)]:
