@@ -349,6 +349,21 @@ attention_decode_kernel(const float* __restrict__ q, const float* __restrict__ k
     cluster.sync();                                            // nobody leaves while its shared memory may still be read
 }
 
+int g_attention_force_split = 0;        // test hook: 0 = automatic, else the cluster size to use (1, 2, 4, 8)
+
+// shared memory of one block that owns Tc keys
+size_t block_smem_bytes(int G, int Tc, int D)
+{
+    return 4 * ((size_t)G * Tc + (size_t)(Tc / kSegKeys) * G * D + 8 + 8 + (size_t)kAttnWarps * G);
+}
+
+// keys per block for a cluster of C blocks: the row's 256-key segments dealt out in equal whole numbers
+int keys_per_block(int T, int C)
+{
+    const int n_seg = (T + kSegKeys - 1) / kSegKeys;
+    return (n_seg + C - 1) / C * kSegKeys;
+}
+
 template <int G, int DC>
 cudaError_t launch_attention_t(const float* q, const float* k, const float* v, float scale, int B, int Hq, int Hkv, int T, int D,
                                float* o, size_t smem, int C, int Tc, cudaStream_t stream)
@@ -366,33 +381,31 @@ cudaError_t launch_attention_t(const float* q, const float* k, const float* v, f
         configured[dev] = true;
     }
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)C, (unsigned)(B * Hkv));
-    cfg.blockDim = dim3(kAttnThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)C;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    for (;;) {
+        cfg.gridDim = dim3((unsigned)C, (unsigned)(B * Hkv));
+        cfg.blockDim = dim3(kAttnThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)C;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        // a cluster this large may not fit where the stream runs (few SMs, a partition): halve it while the scores
+        // of a block still fit (schedule only: same bits)
+        int n_clusters = 0;
+        e = cudaOccupancyMaxActiveClusters(&n_clusters, kern, &cfg);
+        if (e == cudaSuccess && n_clusters >= 1) break;
+        cudaGetLastError();
+        if (C == 1) return e != cudaSuccess ? e : cudaErrorLaunchOutOfResources;
+        C /= 2;
+        Tc = keys_per_block(T, C);
+        smem = block_smem_bytes(G, Tc, D);
+        if (smem > 227u * 1024u) return cudaErrorLaunchOutOfResources;
+    }
     return cudaLaunchKernelEx(&cfg, kern, q, k, v, scale, Hq, Hkv, T, D, Tc, o);
-}
-
-int g_attention_force_split = 0;        // test hook: 0 = automatic, else the cluster size to use (1, 2, 4, 8)
-
-// shared memory of one block that owns Tc keys
-size_t block_smem_bytes(int G, int Tc, int D)
-{
-    return 4 * ((size_t)G * Tc + (size_t)(Tc / kSegKeys) * G * D + 8 + 8 + (size_t)kAttnWarps * G);
-}
-
-// keys per block for a cluster of C blocks: the row's 256-key segments dealt out in equal whole numbers
-int keys_per_block(int T, int C)
-{
-    const int n_seg = (T + kSegKeys - 1) / kSegKeys;
-    return (n_seg + C - 1) / C * kSegKeys;
 }
 
 }  // namespace

@@ -98,6 +98,28 @@ def test_attention_invariance():
             B.det_test_green_stream_destroy(handle)
 
 
+def test_attention_large_clusters_on_few_sms():
+    """A 16-block cluster may not fit the SMs a stream is confined to: the launcher then halves the cluster (schedule
+    only) and the bits stay the same."""
+    q, k, v = make_qkv(1, 4, 1, 16500, 64, seed=5)
+    scale = 0.125
+    want = oracle.attention_decode(q.numpy(), k.numpy(), v.numpy(), scale)
+    try:
+        B.det_test_attention_set_split(16)
+        assert_bits_equal(run_gpu_attention(q, k, v, scale), want, "whole device")
+        for sms in (8, 16):
+            try:
+                stream_ptr, handle, granted = B.det_test_green_stream_create(sms)
+            except B.DetLinearError:
+                continue
+            try:
+                assert_bits_equal(run_gpu_attention(q, k, v, scale, stream=stream_ptr), want, f"{granted} SMs")
+            finally:
+                B.det_test_green_stream_destroy(handle)
+    finally:
+        B.det_test_attention_set_split(0)
+
+
 def test_attention_argument_checks():
     q, k, v = make_qkv(1, 6, 2, 16, 128, seed=1)              # 3 query heads per KV head: not served
     o = torch.empty(1, 6, 128, device="cuda")
